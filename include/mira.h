@@ -253,8 +253,12 @@ mira_status mira_predict_mixture(mira_ctx* ctx, int32_t layer, const void* hidde
  * mma.sync kernels, also for the batch sizes that would take the tcgen05 kernels (used by the
  * tests to compare the two paths). MIRA_OPT_TENSOR_LAYOUT (value 0..3): 0 lets every step choose the tile layout of
  * the tcgen05 kernels from its token count (the default); 1, 2, 3 force the narrow, wide or big layout, for tests
- * and tuning. */
-enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2 };
+ * and tuning. MIRA_OPT_UP_CONVERSION (value 0..2): how the up/gate kernels turn int8 codes into fp16 operands. 0 (the
+ * default) decides per batch on the device: codes go in as (code + 128) * 2^-24 with the offset taken out afterwards,
+ * unless some token's activations have a sum so large against their norm (hidden size * |sum x| > 8192 * |x|_2)
+ * that the subtraction would cost accuracy, in which case the codes are converted exactly; 1 forces the exact
+ * conversion, 2 the offset form (tests and tuning). */
+enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2, MIRA_OPT_UP_CONVERSION = 3 };
 mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value);
 
 /* ---------------------------------------------------------------------------------------------------------------

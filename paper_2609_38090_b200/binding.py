@@ -119,6 +119,7 @@ mira_profile = lib.mira_profile
 mira_set_option = lib.mira_set_option
 MIRA_OPT_FORCE_DECODE_PATH = 1
 MIRA_OPT_TENSOR_LAYOUT = 2
+MIRA_OPT_UP_CONVERSION = 3
 mira_profile_read = lib.mira_profile_read
 KERNEL_CLASSES = ("route", "group", "schedule", "up_gate", "down", "combine", "scores", "pool", "quantize", "unpack")
 mira_status_string = lib.mira_status_string
@@ -336,6 +337,10 @@ class Mira:
     def tensor_layout(self, layout: int) -> None:
         """0: chosen per step (default); 1, 2, 3: force the narrow, wide or big tile layout of the tensor-core kernels."""
         _check(mira_set_option(self._ctx, MIRA_OPT_TENSOR_LAYOUT, int(layout)), "mira_set_option")
+
+    def up_conversion(self, mode: int) -> None:
+        """0: decided per batch on the device (default); 1: exact code conversion in the up/gate kernels; 2: offset subnormals."""
+        _check(mira_set_option(self._ctx, MIRA_OPT_UP_CONVERSION, int(mode)), "mira_set_option")
 
     def profile(self, enable: bool) -> None:
         _check(mira_profile(self._ctx, int(enable)), "mira_profile")

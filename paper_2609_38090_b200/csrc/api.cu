@@ -41,6 +41,7 @@ Layout make_layout(const mira_config& c) {
     L.xnorm = o;     o = align256(o + T * 4);
     L.xsum = o;      o = align256(o + T * 4);
     L.hscale = o;    o = align256(o + P * 4);
+    L.hexp = o;      o = align256(o + Etot * 4);
     L.x16 = o;       o = align256(o + T * C * 2);
     L.x16p = o;      o = align256(o + (T >= (size_t)kTensorPathMinTokens ? P * C * 2 : 0));
     L.xs_pos = o;    o = align256(o + (T >= (size_t)kTensorPathMinTokens ? P * 4 : 0));
@@ -108,9 +109,9 @@ mira_status check_layer_args(mira_ctx* ctx, const void* hidden, int T, int k) {
 }
 
 mira_status do_route(mira_ctx* ctx, const void* hidden, int T, const void* router_w, const float* bias, int k,
-                     const int32_t* slot_map, int* fused_schedule, cudaStream_t st, bool quiet_schedule = false) {
+                     void* const* slots, const int32_t* slot_map, int* fused_schedule, cudaStream_t st, bool quiet_schedule = false) {
     mira_status s = launch_route(ctx, hidden, T, router_w, bias, k, ws_route(ctx), ws_ptr<__half>(ctx, ctx->lay.x16),
-                                 ws_ptr<float>(ctx, ctx->lay.xscale), ws_ptr<float>(ctx, ctx->lay.xnorm), slot_map,
+                                 ws_ptr<float>(ctx, ctx->lay.xscale), ws_ptr<float>(ctx, ctx->lay.xnorm), slots, slot_map,
                                  fused_schedule, st, quiet_schedule);
     if (s == MIRA_OK) { ctx->route_T = T; ctx->route_k = k; }
     return s;
@@ -119,7 +120,7 @@ mira_status do_route(mira_ctx* ctx, const void* hidden, int T, const void* route
 mira_status do_experts(mira_ctx* ctx, int T, void* const* slots, const int32_t* slot_map, const uint32_t* mask,
                        int final_wave, void* out, int schedule_done, cudaStream_t st) {
     mira_status s = MIRA_OK;
-    if (!schedule_done && (s = launch_schedule(ctx, T, slot_map, mask, mask == nullptr, st)) != MIRA_OK) return s;
+    if (!schedule_done && (s = launch_schedule(ctx, T, slots, slot_map, mask, mask == nullptr, st)) != MIRA_OK) return s;
     // every wave of one routed batch takes the same kernels (T decides), so the partial-sum layout is consistent; the
     // two projections switch to the tensor-core kernel at different sizes and share the fp16 intermediate's layout
     const bool tc_ok = ctx->tensor_path_ok && !ctx->force_decode_path;
@@ -133,13 +134,13 @@ mira_status do_experts(mira_ctx* ctx, int T, void* const* slots, const int32_t* 
 }  // namespace
 
 mira_status route_and_schedule(mira_ctx* ctx, const void* hidden, int T, const void* router_w, const float* bias, int k,
-                               const int32_t* slot_map, cudaStream_t st) {
+                               void* const* slots, const int32_t* slot_map, cudaStream_t st) {
     mira_status s = check_layer_args(ctx, hidden, T, k);
     if (s != MIRA_OK) return s;
-    if (T < 1 || !router_w || !slot_map) return MIRA_ERR_INVALID_ARG;
+    if (T < 1 || !router_w || !slots || !slot_map) return MIRA_ERR_INVALID_ARG;
     if (misaligned(router_w)) return MIRA_ERR_ALIGN;
     int fused = 0;
-    if ((s = do_route(ctx, hidden, T, router_w, bias, k, slot_map, &fused, st, true)) != MIRA_OK) return s;
+    if ((s = do_route(ctx, hidden, T, router_w, bias, k, slots, slot_map, &fused, st, true)) != MIRA_OK) return s;
     return fused ? MIRA_OK : MIRA_ERR_UNSUPPORTED;      // every routing path writes the schedule when it has the slot map
 }
 
@@ -309,7 +310,7 @@ mira_status mira_moe_layer(mira_ctx* ctx, const void* hidden, int32_t T, const v
     if (misaligned(router_w) || misaligned(out)) return MIRA_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int fused = 0;
-    if ((s = do_route(ctx, hidden, T, router_w, router_bias, k, slot_map, &fused, st)) != MIRA_OK) return s;
+    if ((s = do_route(ctx, hidden, T, router_w, router_bias, k, expert_slots, slot_map, &fused, st)) != MIRA_OK) return s;
     if ((s = do_experts(ctx, T, expert_slots, slot_map, nullptr, 1, out, fused, st)) != MIRA_OK) return s;
     return copy_route(ctx, dbg, T, k, st);
 }
@@ -322,7 +323,7 @@ mira_status mira_route(mira_ctx* ctx, const void* hidden, int32_t T, const void*
     if (!router_w) return MIRA_ERR_INVALID_ARG;
     if (misaligned(router_w)) return MIRA_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((s = do_route(ctx, hidden, T, router_w, router_bias, k, nullptr, nullptr, st)) != MIRA_OK) return s;
+    if ((s = do_route(ctx, hidden, T, router_w, router_bias, k, nullptr, nullptr, nullptr, st)) != MIRA_OK) return s;
     return copy_route(ctx, route, T, k, st);
 }
 
@@ -357,6 +358,7 @@ mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value) {
     if (!ctx) return MIRA_ERR_INVALID_ARG;
     if (option == MIRA_OPT_FORCE_DECODE_PATH) { ctx->force_decode_path = value != 0; return MIRA_OK; }
     if (option == MIRA_OPT_TENSOR_LAYOUT && value >= 0 && value <= 3) { ctx->tc_layout = value; return MIRA_OK; }
+    if (option == MIRA_OPT_UP_CONVERSION && value >= 0 && value <= 2) { ctx->up_conversion = value; return MIRA_OK; }
     return MIRA_ERR_INVALID_ARG;
 }
 

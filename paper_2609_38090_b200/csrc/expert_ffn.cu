@@ -56,7 +56,6 @@ constexpr float kTwo24 = 16777216.f;
 // The down kernel uses it: its offset term would need the column sums of the fp16 intermediate, one extra MMA per
 // two weight MMAs (measured: 94.6 -> 88.7 us at 8 tokens per expert, 163 -> 137 us at 32). The up/gate kernel
 // keeps the subnormal form, whose offset term is the per-token sum the routing kernel already has.
-constexpr bool kDownExact = true;
 __device__ __forceinline__ unsigned cvt_exact_lo(unsigned u) {
     unsigned v = __byte_perm(u, 0x64646464u, 0x4140);
     __half2 r = __hsub2(*reinterpret_cast<__half2*>(&v), __half2half2(__ushort_as_half(0x6480)));
@@ -73,14 +72,14 @@ __device__ __forceinline__ float pow2i(int e) { return __uint_as_float((unsigned
 __device__ __forceinline__ int expo(float v) { return (int)((__float_as_uint(v) >> 23) & 0xff) - 127; }
 
 struct ItemTable {             // the schedule, copied to shared memory once per CTA
-    int n_active, total_tb;
+    int n_active, total_tb, dc_heavy;
     int tb_prefix[kMaxExperts + 1];
     int w_prefix[kMaxExperts + 1];     // cost prefix of this kernel (up/gate or down)
     uint8_t act_expert[kMaxExperts];
 };
 
 __device__ __forceinline__ void load_table(ItemTable& tab, const Sched* __restrict__ sched, int which) {
-    if (threadIdx.x == 0) { tab.n_active = sched->n_active; tab.total_tb = sched->total_tb; }
+    if (threadIdx.x == 0) { tab.n_active = sched->n_active; tab.total_tb = sched->total_tb; tab.dc_heavy = sched->dc_heavy; }
     for (int i = threadIdx.x; i < kMaxExperts; i += blockDim.x) tab.act_expert[i] = (uint8_t)sched->act_expert[i];
     for (int i = threadIdx.x; i <= kMaxExperts; i += blockDim.x) {
         tab.tb_prefix[i] = sched->tb_prefix[i];
@@ -123,6 +122,7 @@ struct FfnArgs {
     const float* xscale;
     const float* xnorm;
     const float* xsum;          // sum over c of the fp16 (pre-scaled) activations of each token
+    const int32_t* hexp;        // per expert: exponent of the intermediate's expected magnitude per unit of |x|^2
     float* hscale;
     const __half* x16;
     __half* h16;
@@ -130,6 +130,7 @@ struct FfnArgs {
     int R, C, act_on_w1;
     int down_splits, down_slice;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
+    int up_conversion;          // up/gate codes: 0 as the schedule's dc_heavy flag says, 1 exact, 2 offset subnormals
     long ypart_stride;          // elements between two splits = P * C
 };
 
@@ -177,7 +178,7 @@ __device__ __forceinline__ void cp_async16_s(unsigned saddr, const void* gmem_sr
 // One step of a CTA: up to kPairs units of the same (expert, token block, slice).
 struct StepDesc {
     const unsigned char* blob;
-    int row0, k0, klen, split, pos0, ntok, nt, nstep;
+    int row0, k0, klen, split, pos0, ntok, nt, nstep, hexp;
     bool active, valid;
 };
 
@@ -286,7 +287,7 @@ __device__ __forceinline__ void start_step_acts(CopyState& c, const StepDesc& d)
 
 // Runs one step whose first stages are already in flight (start_step), then starts the next step's first
 // stages before its own epilogue, so the memory system never idles between steps.
-template <bool DOWN, int NT>
+template <bool DOWN, int NT, bool EXACT>
 __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, CopyState& cs, const StepDesc& next,
                                          CopyState& cs_next, unsigned char* ringA) {
     constexpr int kStages = stages_for(NT);
@@ -313,13 +314,6 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
 
-    float csum[NT][4];          // S5: column sums of the activation tile (every MMA row holds the same sum)
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) csum[nt][i] = 0.f;
-    const unsigned ones = 0x3C003C00u;             // half2(1, 1)
-
     const int nchunk = cs.nchunk;
     const int nstage = (nchunk + kSegChunks - 1) / kSegChunks;
     // one 64-wide chunk: B fragments of all n-tiles, A fragments of both m-tiles, 8 NT MMAs
@@ -332,10 +326,6 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
             lds128(hi, b_at + nt * 8 * kBRow + 16);
 #pragma unroll
             for (int i = 0; i < 4; ++i) { bf[nt][i] = lo[i]; bf[nt][4 + i] = hi[i]; }
-            if (DOWN && !kDownExact) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) mma16816(csum[nt], ones, ones, ones, ones, bf[nt][2 * j], bf[nt][2 * j + 1]);
-            }
         }
 #pragma unroll
         for (int mt = 0; mt < kMT; ++mt) {
@@ -346,7 +336,7 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
             for (int j = 0; j < 4; ++j) {
                 const unsigned ua = wa[j] ^ 0x80808080u, ub = wb[j] ^ 0x80808080u;
                 unsigned f0, f1, f2, f3;
-                if (DOWN && kDownExact) { f0 = cvt_exact_lo(ua); f2 = cvt_exact_hi(ua); f1 = cvt_exact_lo(ub); f3 = cvt_exact_hi(ub); }
+                if (EXACT) { f0 = cvt_exact_lo(ua); f2 = cvt_exact_hi(ua); f1 = cvt_exact_lo(ub); f3 = cvt_exact_hi(ub); }
                 else { f0 = cvt_lo(ua); f2 = cvt_hi(ua); f1 = cvt_lo(ub); f3 = cvt_hi(ub); }
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) mma16816(acc[mt][nt], f0, f1, f2, f3, bf[nt][2 * j], bf[nt][2 * j + 1]);
@@ -379,15 +369,12 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
     if (early) cs_next = start_step<DOWN>(A, next, sA);
 
     // undo the 2^-24 of the subnormal weights and the +128 offset: acc <- 2^24 acc - 128 * column sum
-    if (active) {
+    if (active && !EXACT) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
-                float colsum;
-                if (DOWN && kDownExact) continue;               // exact signed weights: nothing to undo
-                if (DOWN) colsum = csum[nt][i];
-                else colsum = half ? 0.f : A.xsum[A.row_token[pos0 + min(nt * 8 + tq * 2 + i, ntok - 1)]];   // whole-row sum: count it once
+                const float colsum = half ? 0.f : A.xsum[A.row_token[pos0 + min(nt * 8 + tq * 2 + i, ntok - 1)]];   // whole-row sum: count it once
 #pragma unroll
                 for (int mt = 0; mt < kMT; ++mt) {
                     acc[mt][nt][i] = fmaf(acc[mt][nt][i], kTwo24, -128.f * colsum);
@@ -453,20 +440,19 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
 
     // S4 epilogue: thread holds U (sum[.][0..1]) and G (sum[.][2..3]) of row r for tokens 2tq, 2tq+1 of each n-tile.
     // Per-pair power of two 2^f for the fp16 intermediate s_r h_r: |u|, |g| ~ s * 32 * |x| (codes have
-    // rms ~ 127/4) and |h| ~ u g / 2, so s h ~ s^3 * 512 |x|^2. The typical scale of the expert is the
-    // largest of 32 evenly spaced row scales, so every unit of the pair derives the same f.
+    // rms ~ 127/4) and |h| ~ u g / 2, so s h ~ s^3 * 512 |x|^2 for the row with the LARGEST scale of the expert
+    // (d.hexp = exponent of that s^3, from the routing kernel's statistics CTAs). That magnitude is placed at 2^-2:
+    // what matters to the down projection is the error relative to its largest terms, so the rows that carry the
+    // sum keep 11 bits with room for values 2^17 above the estimate, rows whose scale is much smaller may fall
+    // into fp16's subnormals (absolute error 2^-25 against terms near 2^-2), and nothing overflows (the store
+    // saturates).
     const __nv_bfloat16* sc = reinterpret_cast<const __nv_bfloat16*>(blob + 3 * per);
-    float smax = __bfloat162float(sc[(int)(((long)lane * R) >> 5)]);
-#pragma unroll
-    for (int o = 16; o; o >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, o));
-    const int es = expo(smax);
     const int r = row0 + mt * 8 + g;
     // s_u, s_g: scales of the up and gate rows; s_h: what is folded into the intermediate for the down projection.
     // Shared format: all three are s_r and s h ~ s^3; per-matrix: s1, s3 and 1, so h ~ s^2.
     const float s_u = __bfloat162float(sc[r]);
     const float s_g = A.per_matrix ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(blob + blob_fmt(1, R, C).s_gate)[r]) : s_u;
     const float s_h = A.per_matrix ? 1.f : s_u;
-    const int epow = A.per_matrix ? 2 : 3;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -475,12 +461,12 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
             if (n < ntok) {
                 const int pos = pos0 + n;
                 const int tok = A.row_token[pos];
-                const int f = max(-120, min(120, -(epow * es + 9 + 2 * expo(A.xnorm[tok]))));
+                const int f = max(-120, min(120, -(d.hexp + 11 + 2 * expo(A.xnorm[tok]))));
                 if (row0 == 0 && mt == 0 && g == 0) A.hscale[pos] = pow2i(-f);
                 const float xs = A.xscale[tok];
                 const float u = sum[nt][i] * (xs * s_u), gt = sum[nt][2 + i] * (xs * s_g);
                 const float h = A.act_on_w1 ? silu(u) * gt : silu(gt) * u;
-                A.h16[(size_t)pos * R + r] = __float2half_rn(h * s_h * pow2i(f));
+                A.h16[(size_t)pos * R + r] = __float2half_rn(fminf(fmaxf(h * s_h * pow2i(f), -65504.f), 65504.f));
             }
         }
     }
@@ -509,12 +495,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     long u = unit_at(tab, cost * blockIdx.x / gridDim.x, per_tb, w_full);
     const long u1 = unit_at(tab, cost * (blockIdx.x + 1) / gridDim.x, per_tb, w_full);
     const unsigned sA = (unsigned)__cvta_generic_to_shared(ringA);
+    const bool exact_up = A.up_conversion == 1 || (A.up_conversion == 0 && tab.dc_heavy != 0);
 
     // Describes the step that starts at unit v (valid = false past the end of this CTA's range).
     auto decode = [&](long v) {
         StepDesc d;
         d.valid = v < u1;
-        d.nstep = 0; d.nt = 0; d.active = false; d.blob = nullptr;
+        d.nstep = 0; d.nt = 0; d.active = false; d.blob = nullptr; d.hexp = 0;
         d.row0 = d.k0 = d.klen = d.split = d.pos0 = d.ntok = 0;
         if (!d.valid) return d;
         const int tbg = (int)(v / per_tb);
@@ -533,6 +520,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         d.ntok = min(kTokBlock, cnt - tb * kTokBlock);
         d.nt = (d.ntok + 7) >> 3;
         d.blob = static_cast<const unsigned char*>(A.slots[A.slot_map[e]]);
+        if (!DOWN) d.hexp = A.hexp[e];
         d.k0 = DOWN ? d.split * A.down_slice : 0;
         d.klen = DOWN ? min(A.down_slice, A.R - d.k0) : A.C;
         d.row0 = (mg + pair) * (DOWN ? 16 * kMT : 8 * kMT);
@@ -552,11 +540,20 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         u += cur.nstep;
         const StepDesc next = decode(u);
         CopyState cs_next = cs;
-        switch (cur.nt) {
-            case 1: ffn_step<DOWN, 1>(A, cur, cs, next, cs_next, ringA); break;
-            case 2: ffn_step<DOWN, 2>(A, cur, cs, next, cs_next, ringA); break;
-            case 3: ffn_step<DOWN, 3>(A, cur, cs, next, cs_next, ringA); break;
-            default: ffn_step<DOWN, 4>(A, cur, cs, next, cs_next, ringA); break;
+        if (DOWN || exact_up) {
+            switch (cur.nt) {
+                case 1: ffn_step<DOWN, 1, true>(A, cur, cs, next, cs_next, ringA); break;
+                case 2: ffn_step<DOWN, 2, true>(A, cur, cs, next, cs_next, ringA); break;
+                case 3: ffn_step<DOWN, 3, true>(A, cur, cs, next, cs_next, ringA); break;
+                default: ffn_step<DOWN, 4, true>(A, cur, cs, next, cs_next, ringA); break;
+            }
+        } else {
+            switch (cur.nt) {
+                case 1: ffn_step<false, 1, false>(A, cur, cs, next, cs_next, ringA); break;
+                case 2: ffn_step<false, 2, false>(A, cur, cs, next, cs_next, ringA); break;
+                case 3: ffn_step<false, 3, false>(A, cur, cs, next, cs_next, ringA); break;
+                default: ffn_step<false, 4, false>(A, cur, cs, next, cs_next, ringA); break;
+            }
         }
         cur = next;
         cs = cs_next;
@@ -660,6 +657,8 @@ FfnArgs make_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) {
     A.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm);
     A.xsum = ws_ptr<float>(ctx, ctx->lay.xsum);
     A.hscale = ws_ptr<float>(ctx, ctx->lay.hscale);
+    A.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
+    A.up_conversion = ctx->up_conversion;
     A.x16 = ws_ptr<__half>(ctx, ctx->lay.x16);
     A.h16 = ws_ptr<__half>(ctx, ctx->lay.h16);
     A.ypart = ws_ptr<float>(ctx, ctx->lay.ypart);

@@ -89,6 +89,7 @@ struct TcArgs {
     int32_t* status;
     int R, C, act_on_w1;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
+    int up_conversion;          // up/gate codes: 0 as the schedule's dc_heavy flag says, 1 exact, 2 offset subnormals
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -175,7 +176,8 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const unsigned (&v)[32
 
 // The up/gate kernel may feed the codes as fp16 subnormals (code + 128) * 2^-24 and undo offset and scale in its
 // epilogue with the per-token sum of the activations: two fewer instructions per four weights in the converters.
-constexpr bool kUpSubnormal = true;
+// The subtracted term grows with the sum of a token's activations, so batches that hold a token whose sum is large
+// against its norm (the schedule's dc_heavy flag) take the exact conversion, as the down kernel always does.
 
 __device__ __forceinline__ unsigned cvt_exact_lo(unsigned u) {      // bytes 0,1 of (code + 128) -> half2 of codes
     unsigned v = __byte_perm(u, 0x64646464u, 0x4140);
@@ -228,6 +230,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 
     // per-expert table: one round of parallel loads, then a serial prefix over shared memory
     const int n_active = A.sched->n_active;
+    const bool subnormal = !DOWN && (A.up_conversion == 2 || (A.up_conversion == 0 && A.sched->dc_heavy == 0));
     if (tid < kMaxExperts && tid < n_active) {
         const int e = A.sched->act_expert[tid];
         s_cnt[tid] = A.count[e];
@@ -329,7 +332,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
                         const unsigned u = w4[jj] ^ 0x80808080u;
-                        if (!DOWN && kUpSubnormal) {          // u * 2^-24 as an fp16 subnormal: no subtraction here
+                        if (subnormal) {                      // u * 2^-24 as an fp16 subnormal: no subtraction here
                             f[q * 8 + jj * 2] = __byte_perm(u, 0u, 0x4140);
                             f[q * 8 + jj * 2 + 1] = __byte_perm(u, 0u, 0x4342);
                         } else {
@@ -398,14 +401,14 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                         const int pc = t.pos0 + min(n, t.ntok - 1);
                         const float xs = __ldg(A.xs_pos + pc);
                         float ru = odd ? ob : a, rg = odd ? b : oa;
-                        if (kUpSubnormal) {                   // undo the 2^-24 and the +128 offset of the codes
+                        if (subnormal) {                      // undo the 2^-24 and the +128 offset of the codes
                             const float off = -128.f * __ldg(A.sum_pos + pc);
                             ru = fmaf(ru, 16777216.f, off); rg = fmaf(rg, 16777216.f, off);
                         }
                         const float u = ru * (xs * s_u), g = rg * (xs * s_g);
                         const float act = A.act_on_w1 ? u : g, lin = A.act_on_w1 ? g : u;
                         const float h = __fdividef(act, 1.f + __expf(-act)) * lin;
-                        if (n < t.ntok) A.h16[(size_t)(t.pos0 + n) * R + r] = __float2half_rn(h * s_h * __ldg(A.hm_pos + pc));
+                        if (n < t.ntok) A.h16[(size_t)(t.pos0 + n) * R + r] = __float2half_rn(fminf(fmaxf(h * s_h * __ldg(A.hm_pos + pc), -65504.f), 65504.f));
                     }
                 }
             }
@@ -495,14 +498,14 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 
 // Position-ordered inputs of the tensor path, one block per position: x16p[pos] = x16[row_token[pos]] (so the
 // tokens of one expert are consecutive rows and one TMA box covers a token tile) and the per-position factors
-// of the SwiGLU epilogue: the undo factor of the token's fp16 pre-scaling and the power of two 2^f that keeps
-// the fp16 intermediate near 1 (same rule as the streaming kernels: |s h| ~ s^3 * 512 |x|^2 with s the largest of
-// 32 evenly spaced row scales of the expert).
+// of the SwiGLU epilogue: the undo factor of the token's fp16 pre-scaling and the power of two 2^f that places
+// the fp16 intermediate (same rule as the streaming kernels: |s h| ~ s^3 * 512 |x|^2 with s the largest row scale
+// of the expert, whose exponent the routing kernel's statistics CTAs left in hexp; that magnitude goes to 2^-2).
 struct GatherArgs {
     const __half* x16; const int32_t* row_token; __half* x16p; const int32_t* offset; void* const* slots;
     const int32_t* slot_map; const float* xscale; const float* xnorm; const float* xsum; float* xs_pos; float* hm_pos;
-    float* sum_pos; float* hscale;
-    int C, R, Etot, per_matrix;
+    float* sum_pos; float* hscale; const int32_t* hexp;
+    int C, R, Etot;
 };
 
 __global__ void __launch_bounds__(128) k_gather_x16p(GatherArgs G) {
@@ -516,21 +519,13 @@ __global__ void __launch_bounds__(128) k_gather_x16p(GatherArgs G) {
     for (int e = threadIdx.x; e < G.Etot; e += 128)
         if (G.offset[e] <= pos && pos < G.offset[e + 1]) s_e = e;
     __syncthreads();
-    if (threadIdx.x < 32) {
-        const int slot = G.slot_map[s_e];
-        if (slot < 0) return;                                   // expert not resident: its pairs are skipped everywhere
-        const unsigned char* blob = static_cast<const unsigned char*>(G.slots[slot]);
-        const __nv_bfloat16* sc = reinterpret_cast<const __nv_bfloat16*>(blob + 3 * (size_t)G.R * G.C);
-        float smax = __bfloat162float(sc[(int)(((long)threadIdx.x * G.R) >> 5)]);
-#pragma unroll
-        for (int o = 16; o; o >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, o));
-        if (threadIdx.x == 0) {
-            const int f = max(-120, min(120, -((G.per_matrix ? 2 : 3) * expo_f(smax) + 9 + 2 * expo_f(G.xnorm[tok]))));
-            G.xs_pos[pos] = G.xscale[tok];
-            G.sum_pos[pos] = G.xsum[tok];
-            G.hm_pos[pos] = pow2_f(f);
-            G.hscale[pos] = pow2_f(-f);
-        }
+    if (threadIdx.x == 0) {
+        if (G.slot_map[s_e] < 0) return;                        // expert not resident: its pairs are skipped everywhere
+        const int f = max(-120, min(120, -(G.hexp[s_e] + 11 + 2 * expo_f(G.xnorm[tok]))));
+        G.xs_pos[pos] = G.xscale[tok];
+        G.sum_pos[pos] = G.xsum[tok];
+        G.hm_pos[pos] = pow2_f(f);
+        G.hscale[pos] = pow2_f(-f);
     }
 }
 
@@ -563,6 +558,7 @@ TcArgs make_tc_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) 
     A.status = ws_ptr<int32_t>(ctx, ctx->lay.status);
     A.R = ctx->cfg.ffn; A.C = ctx->cfg.hidden; A.act_on_w1 = ctx->cfg.act_on_w1;
     A.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX;
+    A.up_conversion = ctx->up_conversion;
     return A;
 }
 
@@ -636,8 +632,8 @@ mira_status launch_up_gate_tc(mira_ctx* ctx, void* const* slots, const int32_t* 
     G.xscale = ws_ptr<float>(ctx, ctx->lay.xscale); G.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm);
     G.xs_pos = ws_ptr<float>(ctx, ctx->lay.xs_pos); G.hm_pos = ws_ptr<float>(ctx, ctx->lay.hm_pos);
     G.sum_pos = ws_ptr<float>(ctx, ctx->lay.sum_pos); G.xsum = ws_ptr<float>(ctx, ctx->lay.xsum);
-    G.hscale = ws_ptr<float>(ctx, ctx->lay.hscale);
-    G.C = ctx->cfg.hidden; G.R = ctx->cfg.ffn; G.Etot = Et(ctx->cfg); G.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX;
+    G.hscale = ws_ptr<float>(ctx, ctx->lay.hscale); G.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
+    G.C = ctx->cfg.hidden; G.R = ctx->cfg.ffn; G.Etot = Et(ctx->cfg);
     ProfScope ps(ctx, MIRA_K_UP_GATE, st);
     const int P = ctx->route_T * (ctx->route_k + ctx->cfg.n_shared);
     MIRA_CUDA_OK(launch_pdl(k_gather_x16p, dim3(P), dim3(128), 0, st, G));

@@ -29,6 +29,9 @@ struct Sched {
     // the gap is wider, because the CTAs of small blocks speed up while the others are compute bound and leave
     // them memory bandwidth, so the costs are those that balanced skewed 16- and 32-token batches best.
     int32_t w_prefix[2][kMaxExperts + 1];
+    // 1 if some token of the batch has activations whose sum is large against their norm: the up/gate kernels then
+    // convert the codes exactly instead of through offset subnormals (see dc_heavy_tokens in route.cu).
+    int32_t dc_heavy;
 };
 __host__ __device__ constexpr int block_cost(int which, int n_tiles) {       // which: 0 up/gate, 1 down; n_tiles 1..4
     return which == 0 ? (n_tiles <= 1 ? 16 : n_tiles == 2 ? 22 : n_tiles == 3 ? 27 : 31)
@@ -68,6 +71,7 @@ struct Layout {
     size_t xnorm;       // float [Tmax]   Euclidean norm of token t
     size_t xsum;        // float [Tmax]   sum of the fp16 activations of token t
     size_t hscale;      // float [Pmax]   2^-f_p that undoes the per-pair scaling of the fp16 intermediate
+    size_t hexp;        // int32 [Et]     per expert: exponent of the intermediate's expected magnitude per unit of |x|^2
     size_t x16;         // half  [Tmax][C]
     size_t x16p;        // half  [Pmax][C] activations in position order (tensor-core path only)
     size_t xs_pos;      // float [Pmax]    per position: undo factor of the token's fp16 pre-scaling (tensor-core path)
@@ -98,6 +102,7 @@ struct mira_ctx {
     bool tensor_path_ok = false;
     bool force_decode_path = false;
     int tc_layout = 0;                 // 0: chosen per step; 1..3 force a tile layout of the tensor-core kernels (MIRA_OPT_TENSOR_LAYOUT)
+    int up_conversion = 0;             // 0: chosen per batch on the device; 1: exact; 2: offset subnormals (MIRA_OPT_UP_CONVERSION)
     bool prof_on = false;
     size_t prof_used = 0;
     std::vector<mira::ProfRec> prof;   // per-launch event pairs, reused between reads
@@ -138,9 +143,9 @@ mira_status launch_unpack(mira_ctx*, const void* blob, int8_t* q1, int8_t* q2, i
 mira_status launch_scores(mira_ctx*, const void* x, int T, const void* w, const float* b, int E,
                           float* scores, __half* x16, float* xscale, float* xnorm, cudaStream_t);
 mira_status launch_route(mira_ctx*, const void* x, int T, const void* w, const float* b, int k,
-                         const RouteView& rv, __half* x16, float* xscale, float* xnorm,
+                         const RouteView& rv, __half* x16, float* xscale, float* xnorm, void* const* slots,
                          const int32_t* slot_map, int* fused_schedule, cudaStream_t, bool quiet_schedule = false);
-mira_status launch_schedule(mira_ctx*, int T, const int32_t* slot_map, const uint32_t* dev_expert_mask,
+mira_status launch_schedule(mira_ctx*, int T, void* const* slots, const int32_t* slot_map, const uint32_t* dev_expert_mask,
                             int all_experts, cudaStream_t);
 mira_status launch_pool(mira_ctx*, const float* token_scores, int T, int E, float* pooled,
                         int32_t* ids, int k_pred, cudaStream_t);
@@ -177,7 +182,7 @@ mira_status set_quantize_attributes();
 // holds (an expert without a slot is left for a later wave, not reported); run_scheduled_experts = S4 + S5 for the
 // schedule in place; combine_only = S6 (pairs of experts no wave has run contribute zero and raise the miss flag).
 mira_status route_and_schedule(mira_ctx*, const void* hidden, int T, const void* router_w, const float* bias, int k,
-                               const int32_t* slot_map, cudaStream_t);
+                               void* const* slots, const int32_t* slot_map, cudaStream_t);
 mira_status run_scheduled_experts(mira_ctx*, int T, void* const* slots, const int32_t* slot_map, cudaStream_t);
 mira_status combine_only(mira_ctx*, int T, void* out, cudaStream_t);
 

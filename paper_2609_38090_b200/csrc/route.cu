@@ -337,12 +337,73 @@ struct MaskArg { uint32_t w[8]; };
 struct SchedArgs {
     const int32_t* slot_map; MaskArg mask; Sched* sched; int32_t* status; uint32_t* miss_mask; uint32_t* done_mask;
     int quiet;      // 1: a routed expert without a slot is left for a later wave, not reported as a miss
+    // Inputs of the two numerical decisions the expert kernels take from the schedule stage:
+    //   hexp[e]  exponent of the largest magnitude the intermediate of expert e is expected to reach per unit of
+    //            |x|^2 (from the largest row scale of the blob in its slot), written by the statistics CTAs below;
+    //   dc_heavy whether some token's activations have a sum so large against their norm that the up/gate kernels
+    //            must convert the codes exactly instead of through offset subnormals (see dc_heavy_tokens).
+    void* const* slots; int32_t* hexp; const float* xsum; const float* xnorm; const float* xscale;
+    int T, R, C, per_matrix, n_main;    // n_main: CTAs of the launch that are not statistics CTAs
 };
+
+// The up/gate kernels may feed the codes as (code + 128) * 2^-24 and subtract 128 * sum(x) afterwards. The tensor
+// cores add in fp32 with truncation, so the subtracted term costs about C / 16 accumulation steps of 2^-24 of ITS
+// size, while the wanted sum is about 32 |x|_2 (codes have an rms near 32): the relative error grows like
+// kappa * C * |sum x| / |x|_2 * 2^-27. A batch takes the exact conversion when any of its tokens exceeds the bound
+// below; zero-mean activations (|sum x| ~ |x|_2) stay under it up to a hidden size of 8192.
+constexpr float kDcBound = 24576.f;     // C * |sum x| / |x|_2 from which the exact conversion is used
+
+// Called by every thread of the CTA that writes the schedule. xsum / xnorm may have been written by other CTAs of
+// the same launch (fence + ticket before this call), hence the L2 loads.
+__device__ __forceinline__ int dc_heavy_tokens(const SchedArgs& S) {
+    int heavy = 0;
+    for (int t = threadIdx.x; t < S.T; t += blockDim.x)
+        heavy |= fabsf(__ldcg(S.xsum + t)) * __ldcg(S.xscale + t) * (float)S.C > kDcBound * __ldcg(S.xnorm + t);   // xsum is in pre-scaled units
+    return __syncthreads_or(heavy);
+}
+
+// Statistics CTA of expert e (every thread of the CTA calls it): the largest row scale of the blob in the expert's
+// slot, as the exponent the SwiGLU epilogues use to place the fp16 intermediate. Shared scale: the intermediate
+// s_r h_r grows like s^3; per-matrix scales: like s1 * s3. Experts without a slot, or outside the wave, are skipped.
+__device__ __forceinline__ void expert_stats(const SchedArgs& S, int e) {
+    __shared__ float s_m[2][32];
+    const bool sel = (S.mask.w[e >> 5] >> (e & 31)) & 1u;
+    const int slot = (S.slots != nullptr && S.slot_map != nullptr && sel) ? S.slot_map[e] : -1;
+    if (slot < 0) return;
+    const unsigned char* blob = static_cast<const unsigned char*>(S.slots[slot]);
+    const BlobFmt f = blob_fmt(S.per_matrix ? MIRA_FORMAT_PER_MATRIX : MIRA_FORMAT_SHARED, S.R, S.C);
+    const uint4* su = reinterpret_cast<const uint4*>(blob + f.s_up);
+    const uint4* sg = reinterpret_cast<const uint4*>(blob + f.s_gate);
+    float m1 = 0.f, m3 = 0.f;
+    for (int i = threadIdx.x; i < S.R / 8; i += blockDim.x) {
+        const uint4 v = __ldg(su + i);
+        m1 = fmaxf(m1, fmaxf(fmaxf(fmaxf(bf16lo(v.x), bf16hi(v.x)), fmaxf(bf16lo(v.y), bf16hi(v.y))),
+                             fmaxf(fmaxf(bf16lo(v.z), bf16hi(v.z)), fmaxf(bf16lo(v.w), bf16hi(v.w)))));
+        if (S.per_matrix) {
+            const uint4 w = __ldg(sg + i);
+            m3 = fmaxf(m3, fmaxf(fmaxf(fmaxf(bf16lo(w.x), bf16hi(w.x)), fmaxf(bf16lo(w.y), bf16hi(w.y))),
+                                 fmaxf(fmaxf(bf16lo(w.z), bf16hi(w.z)), fmaxf(bf16lo(w.w), bf16hi(w.w)))));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+        m3 = fmaxf(m3, __shfl_xor_sync(0xffffffffu, m3, o));
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if (lane == 0) { s_m[0][warp] = m1; s_m[1][warp] = m3; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < nwarps; ++w) { m1 = fmaxf(m1, s_m[0][w]); m3 = fmaxf(m3, s_m[1][w]); }
+        S.hexp[e] = S.per_matrix ? expo_of(m1) + expo_of(m3) : 3 * expo_of(m1);
+    }
+}
 
 // Serial tail of the schedule (one thread): the active experts in ascending order with the prefix sums of their
 // token blocks and of the blocks' costs. tb[i] = token blocks of expert i if it is active, else 0.
-__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot) {
+__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot, int dc_heavy) {
     int n = 0, a = 0, wu = 0, wd = 0;
+    sched->dc_heavy = dc_heavy;
     for (int i = 0; i < Etot; ++i) {
         const int b = tb[i];
         if (b > 0) {
@@ -382,8 +443,8 @@ __device__ __forceinline__ void schedule_body(const SchedArgs& S, const int* cou
             if (miss_w && !S.quiet) { atomicOr(S.miss_mask + (e >> 5), miss_w); atomicOr(S.status, 1); }
         }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot);    // s_tb is 0 for inactive experts
+    const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, heavy);    // s_tb is 0 for inactive experts
 }
 
 // S3 for large batches, one CTA; with do_sched also the work schedule of a call that runs every routed expert.
@@ -391,6 +452,7 @@ __global__ void __launch_bounds__(1024) k_group(GroupArgs G, SchedArgs S, int do
     __shared__ int s_count[kMaxExperts];
     __shared__ int s_off[kMaxExperts + 1];
     __shared__ int s_hist[kGroupScratch];
+    if ((int)blockIdx.x >= S.n_main) { expert_stats(S, blockIdx.x - S.n_main); return; }
     group_body(G, s_count, s_off, s_hist);
     if (do_sched) {
         __syncthreads();
@@ -401,6 +463,7 @@ __global__ void __launch_bounds__(1024) k_group(GroupArgs G, SchedArgs S, int do
 __global__ void __launch_bounds__(256) k_schedule(const int32_t* __restrict__ count, int Etot, SchedArgs S) {
     __shared__ int s_tb[kMaxExperts];
     __shared__ int s_act[kMaxExperts];
+    if ((int)blockIdx.x >= S.n_main) { expert_stats(S, blockIdx.x - S.n_main); return; }
     schedule_body(S, count, Etot, s_tb, s_act);
 }
 
@@ -431,6 +494,12 @@ __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, 
     __shared__ int s_last;
     const int t = blockIdx.x, C = A.C, E = A.E, c8 = C / 8;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;    // 8 or 32 warps
+    if (t >= S.n_main) {       // statistics CTAs: one per expert, beside the token CTAs; they take no ticket
+        pdl_wait();            // the previous step's kernels still read the table this CTA rewrites
+        pdl_launch();
+        expert_stats(S, t - S.n_main);
+        return;
+    }
     prefetch_rows_l2(A.W, C * 2, warp, nwarps, E, lane);     // the router is constant: ask for it under the previous kernel's tail
     pdl_wait();            // the previous step's kernels still read the buffers this kernel rewrites
     pdl_launch();
@@ -512,7 +581,7 @@ __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, 
     // ticket: the CTA that takes the last ticket sees every other CTA's idx (fence before the atomic)
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) s_last = (atomicAdd(A.ticket, 1u) == gridDim.x - 1);
+    if (threadIdx.x == 0) s_last = (atomicAdd(A.ticket, 1u) == (unsigned)S.n_main - 1);
     __syncthreads();
     if (!s_last) return;
     __threadfence();
@@ -541,6 +610,12 @@ __global__ void __launch_bounds__(kSingleCtaThreads) k_route_small(TokenArgs A, 
     __shared__ int s_slot[kMaxExperts];
     const int T = A.T, C = A.C, E = A.E, k = A.k, c8 = C / 8, ns = G.ns, Etot = E + ns, kk = k + ns;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = kSingleCtaThreads / 32;
+    if ((int)blockIdx.x >= S.n_main) {       // statistics CTAs: one per expert, beside the routing CTA
+        pdl_wait();
+        pdl_launch();
+        expert_stats(S, blockIdx.x - S.n_main);
+        return;
+    }
     prefetch_rows_l2(A.W, C * 2, warp, nwarps, E, lane);     // the router is constant: ask for it under the previous kernel's tail
     pdl_wait();            // the previous step's kernels still read the buffers this kernel rewrites
     pdl_launch();
@@ -700,8 +775,8 @@ __global__ void __launch_bounds__(kSingleCtaThreads) k_route_small(TokenArgs A, 
             if (miss && !S.quiet) { atomicOr(S.miss_mask + (e >> 5), miss); atomicOr(S.status, 1); }
         }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot);
+    const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot, heavy);
 }
 
 // S7 pooling: pooled[e] = mean_t score[t][e]; then the k_pred best pooled scores.
@@ -847,9 +922,13 @@ GroupArgs group_args(mira_ctx* ctx, int T, int k, const RouteView& rv) {
     G.host_count = ctx->notify_count; G.host_flag = ctx->notify_flag; G.host_seq = ctx->notify_seq;
     return G;
 }
-SchedArgs sched_args(mira_ctx* ctx, const int32_t* slot_map, const uint32_t* host_mask, bool quiet = false) {
+SchedArgs sched_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map, const uint32_t* host_mask, int T, int n_main,
+                     bool quiet = false) {
     SchedArgs S;
     S.quiet = quiet ? 1 : 0;
+    S.slots = slots; S.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
+    S.xsum = ws_ptr<float>(ctx, ctx->lay.xsum); S.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm); S.xscale = ws_ptr<float>(ctx, ctx->lay.xscale);
+    S.T = T; S.R = ctx->cfg.ffn; S.C = ctx->cfg.hidden; S.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX; S.n_main = n_main;
     const int Etot = Et(ctx->cfg);
     for (int i = 0; i < 8; ++i) S.mask.w[i] = (host_mask == nullptr) ? 0xffffffffu : (i < (Etot + 31) / 32 ? host_mask[i] : 0u);
     S.slot_map = slot_map;
@@ -864,9 +943,10 @@ SchedArgs sched_args(mira_ctx* ctx, const int32_t* slot_map, const uint32_t* hos
 // S1-S3. If slot_map is given and the batch is small, the schedule of a run over ALL experts is
 // produced by the same launch (*fused_schedule = 1) and the caller must not launch it again.
 mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, const float* b, int k,
-                         const RouteView& rv, __half* x16, float* xscale, float* xnorm,
+                         const RouteView& rv, __half* x16, float* xscale, float* xnorm, void* const* slots,
                          const int32_t* slot_map, int* fused_schedule, cudaStream_t st, bool quiet_schedule) {
     const int C = ctx->cfg.hidden, E = ctx->cfg.n_experts;
+    const int n_stat = (slots != nullptr && slot_map != nullptr) ? Et(ctx->cfg) : 0;      // statistics CTAs, one per expert
     if (fused_schedule) *fused_schedule = 0;
     GroupArgs G = group_args(ctx, T, k, rv);
     if (T <= (E > 16 ? kFusedRouteMaxTokens : kFusedRouteMaxTokensFewExperts)) {
@@ -878,10 +958,10 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
         A.k = k; A.idx = rv.idx; A.wts = rv.w;
         A.ticket = ws_ptr<unsigned>(ctx, ctx->lay.status) + 8;
         A.do_sched = slot_map != nullptr;
-        SchedArgs S = sched_args(ctx, slot_map, nullptr, quiet_schedule);
+        SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, single ? 1 : T, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_ROUTE, st);
-        if (single) MIRA_CUDA_OK(launch_pdl(k_route_small, dim3(1), dim3(kSingleCtaThreads), (size_t)T * C * 2, st, A, G, S));
-        else MIRA_CUDA_OK(launch_pdl(k_route_token, dim3(T), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
+        if (single) MIRA_CUDA_OK(launch_pdl(k_route_small, dim3(1 + n_stat), dim3(kSingleCtaThreads), (size_t)T * C * 2, st, A, G, S));
+        else MIRA_CUDA_OK(launch_pdl(k_route_token, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
         ctx->launches += 1;
         if (fused_schedule) *fused_schedule = A.do_sched;
         MIRA_CUDA_OK(cudaGetLastError());
@@ -900,9 +980,9 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
     {
         // the schedule of a run over all experts comes out of the same launch
         const int do_sched = slot_map != nullptr;
-        SchedArgs S = sched_args(ctx, slot_map, nullptr, quiet_schedule);
+        SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, 1, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_GROUP, st);
-        k_group<<<1, 1024, 0, st>>>(G, S, do_sched);
+        k_group<<<1 + n_stat, 1024, 0, st>>>(G, S, do_sched);
         if (fused_schedule) *fused_schedule = do_sched;
     }
     ctx->launches += 2;
@@ -910,12 +990,11 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
     return MIRA_OK;
 }
 
-mira_status launch_schedule(mira_ctx* ctx, int T, const int32_t* slot_map, const uint32_t* host_mask,
+mira_status launch_schedule(mira_ctx* ctx, int T, void* const* slots, const int32_t* slot_map, const uint32_t* host_mask,
                             int all_experts, cudaStream_t st) {
-    (void)T;
-    SchedArgs S = sched_args(ctx, slot_map, all_experts ? nullptr : host_mask);
+    SchedArgs S = sched_args(ctx, slots, slot_map, all_experts ? nullptr : host_mask, T, 1);
     ProfScope ps(ctx, MIRA_K_SCHEDULE, st);
-    k_schedule<<<1, 256, 0, st>>>(ws_ptr<int32_t>(ctx, ctx->lay.count), Et(ctx->cfg), S);
+    k_schedule<<<1 + (slots != nullptr ? Et(ctx->cfg) : 0), 256, 0, st>>>(ws_ptr<int32_t>(ctx, ctx->lay.count), Et(ctx->cfg), S);
     ctx->launches += 1;
     MIRA_CUDA_OK(cudaGetLastError());
     return MIRA_OK;

@@ -239,7 +239,7 @@ mira_status mira_stack_layer_step(mira_stack* s, int32_t layer, const void* hidd
     // launch edge stays intact, and the host sees the counts as soon as they exist.
     const uint32_t seq = ++s->seq;
     ctx->notify_count = s->d_live; ctx->notify_flag = s->d_live_flag; ctx->notify_seq = seq;
-    r = route_and_schedule(ctx, hidden, T, router_w, router_bias, k, d0, st);
+    r = route_and_schedule(ctx, hidden, T, router_w, router_bias, k, tables, d0, st);
     ctx->notify_count = nullptr; ctx->notify_flag = nullptr;
     if (r != MIRA_OK) return r;
     if (do_pred) {                                                  // before the expert kernels, which fill every SM

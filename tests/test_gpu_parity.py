@@ -428,10 +428,9 @@ def test_largest_hidden_size_and_top_k(T):
     res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k)
     assert np.array_equal(np.sort(dbg["idx"].cpu().numpy(), axis=1), np.sort(res["idx"], axis=1))   # k = E: every expert
     got = out.cpu().numpy()
-    # A max over a million outputs of only 128 terms each sits in the far tail of the fp16 intermediate's rounding
-    # (2.2e-3 measured): the elementwise gate is taken over as many entries as the other tests check, the row-wise
-    # gate over everything.
-    assert gate_a(got[:8], res["out64"][:8]) <= TOL and gate_c(got, res["out64"]) <= TOL
+    # every row, elementwise and row-wise (at this hidden size the up/gate kernels convert the codes exactly: the
+    # offset form's subtracted term would cost accuracy over 1024 accumulation steps)
+    assert gate_a(got, res["out64"]) <= TOL and gate_c(got, res["out64"]) <= TOL
 
 
 @pytest.mark.parametrize("T", [3, 40, 150])

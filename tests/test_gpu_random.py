@@ -56,11 +56,9 @@ def test_random_layer_configurations(seed):
         got = out.float().cpu().numpy()
         assert np.isfinite(got).all(), desc
         if safe.any():
-            # row-wise gate at the tolerance; the elementwise one is a max over up to 150 k entries of very small layers
-            # (a few dozen terms per output), so it gets twice the bar here
             assert gate_c(got[safe], res["out64"][safe], bf16_output=not fp32) <= 2e-3, desc
             if fp32:
-                assert gate_a(got[safe], res["out64"][safe]) <= 4e-3, desc
+                assert gate_a(got[safe], res["out64"][safe]) <= 2e-3, desc
 
 
 def test_random_waves_with_missing_experts():
@@ -101,7 +99,7 @@ def test_random_waves_with_missing_experts():
         ref = oracle.moe_layer(wl.x, wl.wr, wl.bias, [None if e in missing else wl.blobs[e] for e in range(n_tot)], R, k,
                                n_shared=ns)["out64"]
         got = out.cpu().numpy()
-        assert np.isfinite(got).all() and (not safe.any() or gate_a(got[safe], ref[safe]) <= 4e-3), str(sh)
+        assert np.isfinite(got).all() and (not safe.any() or gate_a(got[safe], ref[safe]) <= 2e-3), str(sh)
 
 
 def test_random_stacks_runtime_against_call_by_call_steps():
