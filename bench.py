@@ -35,9 +35,6 @@ from paper_2609_38090_b200 import inputs  # noqa: E402
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 N_BATCHES = 4          # distinct hidden-state batches rotated over the steps
-# DRAM traffic of the up/gate kernel relative to its algorithmic bytes, from the ncu capture summarised in
-# profiles/k_ffn_mixtral_decode32.md (824.8 MB read + 15.2 MB written for 824.4 MB algorithmic): no wasted re-reads.
-UPGATE_TRAFFIC_RATIO = 1.019
 QUANTIZE_STATS: dict = {}        # filled by build_layer: time and rate of mira_quantize_experts
 
 
@@ -46,13 +43,19 @@ def shape_of(name: str, tokens: int | None) -> inputs.LayerShape:
     return base.with_tokens(tokens if tokens else base.T)
 
 
-def peaks() -> tuple[float, float, str]:
-    """(HBM GB/s, bf16 TFLOP/s, source) -- measured on this machine if the file exists."""
+NOMINAL_HBM_GBS = 8000.0       # the vendor's figure the benchmark spec quotes; fractions of it are reported beside the measured ones
+NOMINAL_TFLOPS = 2250.0        # dense bf16 / fp16 tensor rate of the data sheet
+
+
+def peaks() -> tuple[float, float, float, str]:
+    """(HBM GB/s, bf16 TFLOP/s sustained, bf16 TFLOP/s burst, source) -- measured on this machine if the file exists.
+    The copy rate and the cuBLAS rates were taken with torch on this machine's B200s; the sustained rate is under the
+    power cap (SM clock near 1.34 GHz), the burst rate is a short run at full clock."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), "measured"
-    return 6650.0, 1400.0, "fallback"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), float(d.get("bf16_tflops", d["bf16_tflops_sustained"])), "measured"
+    return 6650.0, 1400.0, 1590.0, "fallback"
 
 
 class ClockSampler:
@@ -257,73 +260,13 @@ def replica_throughput(tokens: int, steps: int, world: int, ms_total: float) -> 
     return world * tokens * steps / (ms_total / 1e3)
 
 
-def run_cuda(args):
+def timed_blocks(fn, steps, barrier, dev, world, min_seconds=0.5, finish=None, max_blocks=400):
+    """Times blocks of exactly `steps` steps, each bracketed by barrier + synchronize on both sides and CUDA events
+    on the launching stream, repeated until the blocks together last at least `min_seconds` (so that the clock
+    sampler sees the timed region). Returns the per-block times in ms (max over ranks)."""
     import torch
-    import torch.distributed as dist
-    from paper_2609_38090_b200 import binding
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    dev = torch.device("cuda", local)
-    torch.cuda.set_device(dev)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    sh = shape_of(args.workload, args.tokens)
-    m, blobs, slots, slot_map, wr, bias, xs_host = build_layer(sh, dev)
-    xs = [x.to(dev) for x in xs_host]
-    xs_pinned = [x.pin_memory() for x in xs_host]
-    out = torch.empty((sh.T, sh.C), dtype=torch.bfloat16, device=dev)
-    out_host = torch.empty((sh.T, sh.C), dtype=torch.bfloat16).pin_memory()
-    x_dev = torch.empty((sh.T, sh.C), dtype=torch.bfloat16, device=dev)
-
-    # routing statistics of the rotating batches (untimed): which experts each step touches
-    counts = []
-    for x in xs:
-        r = m.route(x, wr, bias, sh.k)
-        counts.append(r["count"].cpu().tolist())
-    bytes_layer = [algorithmic_bytes(sh, c)[0] for c in counts]
-    bytes_upgate = [algorithmic_bytes(sh, c)[1] for c in counts]
-
-    def step(i):
-        m.moe_layer(xs[i % N_BATCHES], wr, bias, slots, slot_map, sh.k, out=out)
-
-    # End to end: every step copies its hidden states from pinned host memory and its output back. The copies run on
-    # their own streams with two buffers each, so the copy of step i + 1 and the read-back of step i - 1 overlap
-    # the kernels of step i, as a serving loop would arrange it; every step still moves its own bytes.
-    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-    s_main = torch.cuda.current_stream(dev)
-    x_buf = [torch.empty_like(x_dev) for _ in range(2)]
-    o_buf = [torch.empty_like(out) for _ in range(2)]
-    o_host = [torch.empty((sh.T, sh.C), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-    ev_in = [torch.cuda.Event() for _ in range(2)]
-    ev_cmp = [torch.cuda.Event() for _ in range(2)]
-    ev_out = [torch.cuda.Event() for _ in range(2)]
-    for b in range(2):
-        ev_cmp[b].record(s_main); ev_out[b].record(s_main)
-
-    def step_e2e(i):
-        b = i & 1
-        s_in.wait_event(ev_cmp[b])                  # the kernels that read this input buffer two steps ago are done
-        with torch.cuda.stream(s_in):
-            x_buf[b].copy_(xs_pinned[i % N_BATCHES], non_blocking=True)
-            ev_in[b].record(s_in)
-        s_main.wait_event(ev_in[b])
-        s_main.wait_event(ev_out[b])                # this output buffer has been read back
-        m.moe_layer(x_buf[b], wr, bias, slots, slot_map, sh.k, out=o_buf[b])
-        ev_cmp[b].record(s_main)
-        s_out.wait_event(ev_cmp[b])
-        with torch.cuda.stream(s_out):
-            o_host[b].copy_(o_buf[b], non_blocking=True)
-            ev_out[b].record(s_out)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
-    def timed(fn, steps, finish=None):
+    blocks, total = [], 0.0
+    while True:
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         a.record()
@@ -333,34 +276,213 @@ def run_cuda(args):
             finish()                                # e.g. make the stop event wait for copies on other streams
         b.record()
         barrier()
-        return reduce_max_ms(a.elapsed_time(b), dev, world)
+        ms = reduce_max_ms(a.elapsed_time(b), dev, world)
+        blocks.append(ms)
+        total += ms
+        if total >= 1e3 * min_seconds or len(blocks) >= max_blocks:
+            return blocks
 
-    sampler = ClockSampler(local) if rank == 0 else None
-    if sampler:
-        sampler.wait_started()
-    for i in range(args.warmup):
+
+def block_stats(blocks, steps):
+    med = statistics.median(blocks)
+    return {"ms_per_step": med / steps, "ms_per_step_best": min(blocks) / steps, "blocks": len(blocks),
+            "timed_seconds": sum(blocks) / 1e3}
+
+
+def clock_record(sampler, lo, hi, ms_per_step):
+    """Clock summary of the samples taken inside one timed region, plus time x clock (ms x MHz) so that steps timed
+    at different clocks can be compared."""
+    if sampler is None:
+        return None
+    c = sampler.summary(lo, hi) if hi > lo else sampler.summary(lo, max(sampler.mark(), lo + 1))
+    c["samples_in_timed_region"] = max(hi - lo, 0)
+    c["ms_per_step_x_sm_mhz"] = (ms_per_step * c["sm_mhz"]) if c.get("sm_mhz") else None
+    return c
+
+
+def traffic_ratio(key: str):
+    """DRAM bytes of one launch relative to its algorithmic bytes, from the ncu capture summarised under profiles/
+    (profiles/traffic_ratios.json, written when the capture is taken); None if no capture is on record."""
+    p = os.path.join(ROOT, "profiles", "traffic_ratios.json")
+    try:
+        return json.load(open(p)).get(key)
+    except (OSError, ValueError):
+        return None
+
+
+class ResidentLayer:
+    """One resident MoE layer on the device (all experts in their slots), shared by the token counts timed on it."""
+
+    def __init__(self, sh: inputs.LayerShape, dev):
+        self.sh, self.dev = sh, dev
+        self.m0, self.blobs, self.slots, self.slot_map, self.wr, self.bias, _ = build_layer(sh, dev)
+        self.quantize = dict(QUANTIZE_STATS)
+
+    def context(self, T):
+        from paper_2609_38090_b200 import binding
+        sh = self.sh
+        return binding.Mira(sh.C, sh.R, sh.E, n_shared=sh.n_shared, n_layers=32, max_tokens=T, max_top_k=sh.k,
+                            device=self.dev, fmt=FMT)
+
+
+def measure_resident(layer: ResidentLayer, T: int, args, world, rank, sampler, barrier, e2e=True):
+    """Times one token count of a resident layer: the steps with inputs in HBM (blocks of args.steps steps for at
+    least half a second), the same steps end to end (H2D of the hidden states, D2H of the output, every step), and a
+    per-kernel pass with CUDA events around every launch. Returns the record of this configuration."""
+    import torch
+    sh, dev = layer.sh.with_tokens(T), layer.dev
+    m = layer.context(T)
+    wr, bias, slots, slot_map = layer.wr, layer.bias, layer.slots, layer.slot_map
+    xs_host = [torch.from_numpy(inputs.hidden(sh, T, step=i)).to(torch.bfloat16) for i in range(N_BATCHES)]
+    xs = [x.to(dev) for x in xs_host]
+    out = torch.empty((T, sh.C), dtype=torch.bfloat16, device=dev)
+    counts = [m.route(x, wr, bias, sh.k)["count"].cpu().tolist() for x in xs]
+    bytes_layer = [algorithmic_bytes(sh, c)[0] for c in counts]
+    bytes_upgate = [algorithmic_bytes(sh, c)[1] for c in counts]
+
+    def step(i):
+        m.moe_layer(xs[i % N_BATCHES], wr, bias, slots, slot_map, sh.k, out=out)
+
+    for i in range(max(args.warmup, 3)):
         step(i)
     barrier()
     launches0 = m.kernel_launches
     lo = sampler.mark() if sampler else 0
-    ms_total = timed(step, args.steps)
+    blocks = timed_blocks(step, args.steps, barrier, dev, world)
     hi = sampler.mark() if sampler else 0
-    launches = m.kernel_launches - launches0
+    launches = (m.kernel_launches - launches0) // len(blocks)
     code, missing = m.poll_status()
     assert code == 0, f"device status {code}, missing experts {missing}"
+    st = block_stats(blocks, args.steps)
+    ms_step = st["ms_per_step"]
+    rec = {"workload": workload_config(sh)["workload"], "tokens": T, **st,
+           "tokens_per_s": replica_throughput(T, 1, world, ms_step), "gpu_launches": int(launches),
+           "clocks": clock_record(sampler, lo, hi, ms_step)}
 
-    for i in range(args.warmup):
-        step_e2e(i)
-    ms_e2e = timed(step_e2e, args.steps, finish=lambda: [s_main.wait_event(e) for e in ev_out])
+    if e2e:
+        # End to end: every step copies its hidden states from pinned host memory and its output back. The copies run
+        # on their own streams with two buffers each, so the copy of step i + 1 and the read-back of step i - 1
+        # overlap the kernels of step i, as a serving loop would arrange it; every step still moves its own bytes.
+        xs_pinned = [x.pin_memory() for x in xs_host]
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        s_main = torch.cuda.current_stream(dev)
+        x_buf = [torch.empty((T, sh.C), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        o_buf = [torch.empty_like(out) for _ in range(2)]
+        o_host = [torch.empty((T, sh.C), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_cmp = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+        for b in range(2):
+            ev_cmp[b].record(s_main); ev_out[b].record(s_main)
 
-    # profiled pass: the same steps with per-kernel events, for the roofline of the dominant kernel
+        def step_e2e(i):
+            b = i & 1
+            s_in.wait_event(ev_cmp[b])              # the kernels that read this input buffer two steps ago are done
+            with torch.cuda.stream(s_in):
+                x_buf[b].copy_(xs_pinned[i % N_BATCHES], non_blocking=True)
+                ev_in[b].record(s_in)
+            s_main.wait_event(ev_in[b])
+            s_main.wait_event(ev_out[b])            # this output buffer has been read back
+            m.moe_layer(x_buf[b], wr, bias, slots, slot_map, sh.k, out=o_buf[b])
+            ev_cmp[b].record(s_main)
+            s_out.wait_event(ev_cmp[b])
+            with torch.cuda.stream(s_out):
+                o_host[b].copy_(o_buf[b], non_blocking=True)
+                ev_out[b].record(s_out)
+
+        for i in range(max(args.warmup, 3)):
+            step_e2e(i)
+        eb = timed_blocks(step_e2e, args.steps, barrier, dev, world, finish=lambda: [s_main.wait_event(e) for e in ev_out])
+        est = block_stats(eb, args.steps)
+        rec["e2e"] = {"value": world * T / (est["ms_per_step"] / 1e3), "unit": UNIT, "h2d_bytes_per_step": T * sh.C * 2,
+                      "d2h_bytes_per_step": T * sh.C * 2, "ms_per_step": est["ms_per_step"], "blocks": est["blocks"]}
+
+    # per-kernel pass: the same steps with an event pair around every launch (the events switch the programmatic
+    # launch overlap off, so the kernel times add up to a little more than the step)
+    n_prof = max(args.steps, min(400, int(0.1e3 / max(ms_step, 1e-3))))
     m.profile(True)
     barrier()
-    for i in range(args.steps):
+    for i in range(n_prof):
         step(i)
     prof = m.profile_read()
     m.profile(False)
     barrier()
+
+    hbm, tf_sus, tf_burst, src = peaks()
+    tc_kernels = T >= (32 if sh.E + sh.n_shared > 16 else 56)        # up/gate on the tcgen05 grouped GEMM kernel
+    pairs_avg = sum(sum(c) for c in counts) / len(counts)
+    flops_step = 6.0 * sh.R * sh.C * pairs_avg
+    bytes_step = sum(bytes_layer) / len(bytes_layer)
+    tensor_path = tc_kernels and flops_step / (tf_sus * 1e12) > bytes_step / (hbm * 1e9)
+    up_ms, up_n = prof.get("up_gate", (0.0, 0))
+    up_bytes = sum(bytes_upgate) / len(bytes_upgate)
+    up_us = 1e3 * up_ms / max(up_n, 1)
+    total_prof_ms = sum(v[0] for v in prof.values())
+    shares = {k: round(v[0] / total_prof_ms, 4) for k, v in prof.items()} if total_prof_ms else None
+    avg_us = {k: round(1e3 * v[0] / v[1], 2) for k, v in prof.items() if v[1]}
+    if tensor_path:
+        up_flops = 4.0 * sh.R * sh.C * pairs_avg                      # up + gate projections of every pair
+        ach = up_flops / (up_us / 1e6) / 1e12 if up_us > 0 else None
+        rec["roofline"] = {"bound": "tensor", "kernel": "k_ffn_tc<up/gate> (tcgen05 grouped GEMM on in-register dequantized fp16 tiles, SwiGLU epilogue)",
+                           "achieved": ach, "peak": tf_sus, "unit": "TFLOP/s", "frac": (ach / tf_sus) if ach else None,
+                           "frac_of_burst_peak": (ach / tf_burst) if ach else None,
+                           "frac_of_nominal_2250TFLOPs": (ach / NOMINAL_TFLOPS) if ach else None,
+                           "peak_source": src + " (cuBLAS bf16, sustained under the power cap; fp16 has the same nominal rate)",
+                           "traffic": None, "avg_launch_us": up_us, "algorithmic_flops_per_launch": up_flops,
+                           "kernel_share": shares, "kernel_avg_us": avg_us}
+    else:
+        ach = up_bytes / (up_us / 1e6) / 1e9 if up_us > 0 else None
+        key = "k_ffn_up_gate" if not tc_kernels else "k_ffn_tc_up_gate"
+        tr = traffic_ratio(key)
+        rec["roofline"] = {"bound": "hbm", "kernel": ("k_ffn_tc<up/gate> (tcgen05 grouped GEMM, in-register dequant, SwiGLU epilogue)" if tc_kernels
+                                                      else "k_ffn<up/gate> (fused int8 unpack/dequant + up/gate GEMV/GEMM + SwiGLU)"),
+                           "achieved": ach, "peak": hbm, "unit": "GB/s", "frac": (ach / hbm) if ach else None,
+                           "frac_of_nominal_8TBps": (ach / NOMINAL_HBM_GBS) if ach else None, "peak_source": src,
+                           "traffic": (tr["ratio"] * up_bytes) if tr else None,
+                           "traffic_source": (tr["source"] if tr else "no ncu capture of this kernel on record"),
+                           "avg_launch_us": up_us, "algorithmic_bytes_per_launch": up_bytes,
+                           "kernel_share": shares, "kernel_avg_us": avg_us}
+    layer_gbs = bytes_step / (ms_step / 1e3) / 1e9
+    rec["layer_roofline"] = {"bound": "hbm", "algorithmic_bytes_per_step": bytes_step, "achieved": layer_gbs, "peak": hbm,
+                             "unit": "GB/s", "frac": layer_gbs / hbm, "frac_of_nominal_8TBps": layer_gbs / NOMINAL_HBM_GBS,
+                             "peak_source": src,
+                             "active_experts_per_batch": [int(sum(1 for c in cs if c > 0)) for cs in counts]}
+    tfl = flops_step / (ms_step / 1e3) / 1e12
+    rec["layer_tensor"] = {"algorithmic_flops_per_step": flops_step, "achieved": tfl, "unit": "TFLOP/s",
+                           "peak": tf_sus, "frac": tfl / tf_sus, "frac_of_burst_peak": tfl / tf_burst,
+                           "frac_of_nominal_2250TFLOPs": tfl / NOMINAL_TFLOPS, "peak_source": src,
+                           "binding": "tensor" if tensor_path else "hbm"}
+    rec["_m"] = m
+    rec["_xs"] = xs
+    return rec
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sh = shape_of(args.workload, args.tokens)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.wait_started()
+    layer = ResidentLayer(sh, dev)
+    head = measure_resident(layer, sh.T, args, world, rank, sampler, barrier)
+    m, xs = head.pop("_m"), head.pop("_xs")
+    wr, bias = layer.wr, layer.bias
+
     # S7 and S0 carry no target; their times are reported next to the layer's
     pw_np, pb_np = inputs.predictor(sh)
     pred_w = torch.from_numpy(pw_np).to(torch.bfloat16).to(dev)
@@ -389,72 +511,46 @@ def run_cuda(args):
     mprof = m.profile_read()
     m.profile(False)
     mixture_us = 1e3 * sum(v[0] for v in mprof.values()) / 20
-    clocks = None
-    if sampler:
-        # the timed region of a decode step is a few ms, shorter than one sampling period: the window also covers
-        # the end-to-end and the per-kernel passes, which run the same steps back to back
-        clocks = sampler.summary(lo, max(sampler.mark(), lo + 1))
-        clocks["samples_in_timed_region"] = max(hi - lo, 0)
-        clocks["window"] = "timed + end-to-end + per-kernel passes of the same steps"
-        sampler.stop()
 
+    # The other configurations of the workload list, one record each (skipped with --headline-only, with a workload
+    # or token count chosen on the command line, and on multi-GPU launches, where every rank is a replica of the
+    # headline step).
+    others = []
+    default_run = args.workload == "mixtral" and args.tokens is None and not FMT
+    if default_run and world == 1 and not args.headline_only:
+        for T in (1, 8, 2048):
+            r = measure_resident(layer, T, args, world, rank, sampler, barrier, e2e=False)
+            r.pop("_m"); r.pop("_xs")
+            others.append(r)
+        del m, xs
+        others.append(staged_record(args, layer, sampler, barrier, dev, world, rank))
+        del layer
+        torch.cuda.empty_cache()
+        fine = ResidentLayer(inputs.FINE, dev)
+        for T in (4, 64, 1024):
+            r = measure_resident(fine, T, args, world, rank, sampler, barrier, e2e=False)
+            r.pop("_m"); r.pop("_xs")
+            others.append(r)
+        del fine
+        torch.cuda.empty_cache()
+        others.append(stack_record(args, sampler, barrier, dev, world, rank, steps=max(args.steps, 8)))
+    if sampler:
+        sampler.stop()
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    hbm, tflops, src = peaks()
-    # the up/gate projection takes the tcgen05 grouped GEMM kernel from 56 tokens (32 with more than 16 experts)
-    tc_kernels = sh.T >= (32 if sh.E + sh.n_shared > 16 else 56)
-    flops_step = 6.0 * sh.R * sh.C * sum(sum(c) for c in counts) / len(counts)
-    # which roofline binds the step: algorithmic flops at the tensor peak or algorithmic bytes at the HBM peak
-    tensor_path = tc_kernels and flops_step / (tflops * 1e12) > (sum(bytes_layer) / len(bytes_layer)) / (hbm * 1e9)
-    ms_step = ms_total / args.steps
-    value = replica_throughput(sh.T, args.steps, world, ms_total)
-    e2e_value = replica_throughput(sh.T, args.steps, world, ms_e2e)
-    step_bytes = [bytes_layer[i % N_BATCHES] for i in range(args.steps)]
-    up_bytes = [bytes_upgate[i % N_BATCHES] for i in range(args.steps)]
-    up_ms, up_n = prof.get("up_gate", (0.0, 0))
-    achieved = (sum(up_bytes) / max(up_n, 1)) / (up_ms / max(up_n, 1) / 1e3) / 1e9 if up_ms > 0 else None
-    total_prof_ms = sum(v[0] for v in prof.values())
-    roofline = {"bound": "hbm", "kernel": ("k_ffn_tc<up/gate> (tcgen05 grouped GEMM, in-register dequant, SwiGLU epilogue)" if tc_kernels
-                                           else "k_up_gate (fused int8 unpack/dequant + up/gate GEMV/GEMM + SwiGLU)"),
-                "achieved": achieved, "peak": hbm, "unit": "GB/s",
-                "frac": (achieved / hbm) if achieved else None, "peak_source": src,
-                "traffic": None if tc_kernels else UPGATE_TRAFFIC_RATIO * sum(up_bytes) / len(up_bytes),
-                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch, scaled by algorithmic bytes",
-                "avg_launch_us": 1e3 * up_ms / max(up_n, 1),
-                "algorithmic_bytes_per_launch": sum(up_bytes) / len(up_bytes),
-                "kernel_share": {k: round(v[0] / total_prof_ms, 4) for k, v in prof.items()} if total_prof_ms else None,
-                "kernel_avg_us": {k: round(1e3 * v[0] / v[1], 2) for k, v in prof.items()}}
-    if tensor_path:
-        pairs = [sum(counts[i % N_BATCHES]) for i in range(args.steps)]
-        up_flops = [4.0 * sh.R * sh.C * p for p in pairs]                # up + gate projections of every pair
-        ach = (sum(up_flops) / max(up_n, 1)) / (up_ms / max(up_n, 1) / 1e3) / 1e12 if up_ms > 0 else None
-        roofline = {"bound": "tensor", "kernel": "k_ffn_tc<up/gate> (tcgen05 grouped GEMM on in-register dequantized fp16 tiles, SwiGLU epilogue)",
-                    "achieved": ach, "peak": tflops, "unit": "TFLOP/s", "frac": (ach / tflops) if ach else None,
-                    "peak_source": src + " (cuBLAS bf16, sustained; fp16 has the same nominal rate)", "traffic": None,
-                    "avg_launch_us": 1e3 * up_ms / max(up_n, 1), "algorithmic_flops_per_launch": sum(up_flops) / len(up_flops),
-                    "kernel_share": roofline["kernel_share"], "kernel_avg_us": roofline["kernel_avg_us"]}
-    layer_gbs = (sum(step_bytes) / len(step_bytes)) / (ms_step / 1e3) / 1e9
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "metric": METRIC, "value": head["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "ms_per_step_best_block": head["ms_per_step_best"],
+        "timed_blocks": head["blocks"], "timed_seconds": head["timed_seconds"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "s8 weights x f16 activations, f32 accumulate",
         "data": "synthetic", "config": workload_config(sh),
-        "roofline": roofline,
-        "layer_roofline": {"bound": "hbm", "algorithmic_bytes_per_step": sum(step_bytes) / len(step_bytes),
-                           "achieved": layer_gbs, "peak": hbm, "unit": "GB/s", "frac": layer_gbs / hbm,
-                           "frac_of_nominal_8TBps": layer_gbs / 8000.0, "peak_source": src,
-                           "active_experts_per_batch": [int(sum(1 for c in cs if c > 0)) for cs in counts]},
-        "layer_tensor": ({"algorithmic_flops_per_step": 6.0 * sh.R * sh.C * sum(sum(c) for c in counts) / len(counts),
-                          "achieved": 6.0 * sh.R * sh.C * sum(sum(c) for c in counts) / len(counts) / (ms_step / 1e3) / 1e12,
-                          "peak": tflops, "unit": "TFLOP/s",
-                          "frac": 6.0 * sh.R * sh.C * sum(sum(c) for c in counts) / len(counts) / (ms_step / 1e3) / 1e12 / tflops,
-                          "peak_source": src} if tensor_path else None),
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": sh.T * sh.C * 2,
-                "d2h_bytes_per_step": sh.T * sh.C * 2, "ms_per_step": ms_e2e / args.steps},
-        "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": head["roofline"], "layer_roofline": head["layer_roofline"], "layer_tensor": head["layer_tensor"],
+        "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],
+        "timing_note": ("ms_per_step is the median over blocks of exactly --steps steps, each block bracketed by barrier + "
+                        "synchronize and timed with CUDA events, repeated until the blocks last 0.5 s; gpu_launches counts one block"),
         "other_steps": {"predictor_us_per_call": predict_us,
                         "predictor_note": "device time of mira_predict on one batch: linear head, mean over tokens, top-2 (S7)",
                         "mixture_head_us_per_call": mixture_us,
@@ -463,6 +559,8 @@ def run_cuda(args):
                         "quantize_gbs": QUANTIZE_STATS.get("gbs"),
                         "quantize_note": "mira_quantize_experts (S0): fp32 W2 read twice, W1 and W3 once, blob written"},
     }
+    if others:
+        line["configs"] = others
     if world == 1 and not args.no_cpu_baseline:
         # whole batches of the workload until about 10 s of CPU time (large batches: a 64-token slice of each)
         n_tok = min(sh.T, 64)
@@ -474,27 +572,19 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
-def run_staged(args):
+def staged_record(args, layer, sampler, barrier, dev, world, rank):
     """Prefill with the predictor and a small expert cache (the third workload): per step the predictor scores the
     tokens (S7), the router runs (S1-S3), the host reads the expert counts, the experts in the HOT slots run as the
     first wave while the side stream copies the missing experts from pinned host memory into the STAGE slots (S8),
-    and the staged experts run as later waves; the last wave combines. One GPU; ranks > 0 of a multi-GPU launch
-    run the same step as independent replicas."""
+    and the staged experts run as later waves; the last wave combines. Returns the record of the configuration."""
     import torch
-    import torch.distributed as dist
     from paper_2609_38090_b200 import binding
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    dev = torch.device("cuda", local)
-    torch.cuda.set_device(dev)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    sh = shape_of("mixtral", args.tokens or 2048)
+    sh = layer.sh.with_tokens(args.tokens or 2048) if args.mode == "staged" else layer.sh.with_tokens(2048)
     n_hot, n_stage, k_pred = 4, 2, 2
-    m, blobs, slots_all, slot_map_all, wr, bias, xs_host = build_layer(sh, dev)
-    xs = [x.to(dev) for x in xs_host]
+    m = layer.context(sh.T)
+    blobs, wr, bias = layer.blobs, layer.wr, layer.bias
+    xs = [torch.from_numpy(inputs.hidden(sh, sh.T, step=i)).to(torch.bfloat16).to(dev) for i in range(N_BATCHES)]
     E = sh.E
     counts = [m.route(x, wr, bias, sh.k)["count"].cpu().tolist() for x in xs]
     popularity = np.sum(np.array(counts), axis=0)
@@ -505,8 +595,6 @@ def run_staged(args):
     cache = torch.empty((n_hot + n_stage, m.expert_bytes), dtype=torch.uint8, device=dev)
     for i, e in enumerate(hot):
         cache[i].copy_(blobs[e])
-    del blobs, slots_all
-    torch.cuda.empty_cache()
     slots = binding.slot_table(cache)
 
     def smap(pairs):
@@ -560,11 +648,6 @@ def run_staged(args):
             if wi + 1 < len(waves):
                 stage(waves[wi + 1])
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
     # plain pinned host -> device copy rate of this machine, same size as one expert
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     scratch = torch.empty(m.expert_bytes, dtype=torch.uint8, device=dev)
@@ -595,60 +678,44 @@ def run_staged(args):
         return 1e3 * a.elapsed_time(b) / reps                        # us per expert
     scale_shared_us, scale_three_us = scale_copies([0]), scale_copies([0, 1, 2])
 
-    sampler = ClockSampler(local) if rank == 0 else None
-    if sampler:
-        sampler.wait_started()
-    for i in range(args.warmup):
+    for i in range(max(args.warmup, 3)):
         step(i)
     barrier()
     launches0 = m.kernel_launches
     staged_bytes[0] = 0
     lo = sampler.mark() if sampler else 0
-    a.record()
-    for i in range(args.steps):
-        step(i)
-    b.record()
-    barrier()
-    ms_total = reduce_max_ms(a.elapsed_time(b), dev, world)
-    launches = m.kernel_launches - launches0
-    bytes_staged = staged_bytes[0] / args.steps
+    blocks = timed_blocks(step, args.steps, barrier, dev, world)
+    hi = sampler.mark() if sampler else 0
+    st = block_stats(blocks, args.steps)
+    ms_step = st["ms_per_step"]
+    launches = (m.kernel_launches - launches0) // len(blocks)
+    bytes_staged = staged_bytes[0] / (args.steps * len(blocks))
     code, missing = m.poll_status()
     assert code == 0, f"device status {code}, missing experts {missing}"
-    # compute-only time of the same waves (experts already in place): the part staging has to hide behind
+    # compute-only time of the same waves: the part staging has to hide behind
+    n_prof = min(args.steps, 5)
     m.profile(True)
-    for i in range(min(args.steps, 5)):
+    for i in range(n_prof):
         step(i)
     barrier()
     prof = m.profile_read()
     m.profile(False)
-    clocks = None
-    if sampler:
-        clocks = sampler.summary(lo, max(sampler.mark(), lo + 1))
-        sampler.stop()
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    hbm, tflops, src = peaks()
-    ms_step = ms_total / args.steps
-    n_prof = min(args.steps, 5)
+    hbm, tf_sus, tf_burst, src = peaks()
     kernel_ms = sum(v[0] for v in prof.values()) / n_prof
     up_ms, up_n = prof.get("up_gate", (0.0, 1))
     pairs = float(np.mean([sum(c) for c in counts]))
     up_flops = 4.0 * sh.R * sh.C * pairs
     ach = up_flops / (up_ms / n_prof / 1e3) / 1e12 if up_ms > 0 else None
-    cfg = workload_config(sh)
-    cfg["workload"] = (f"{sh.name} layer, prefill {sh.T} tokens with the two-layers-ahead predictor scored per token; "
-                       f"cache of {n_hot} HOT + {n_stage} STAGE slots for {E} experts, the other experts are staged "
-                       "from pinned host memory every step and run as later waves")
-    cfg["hot_experts"] = hot
-    line = {
-        "metric": METRIC, "value": replica_throughput(sh.T, args.steps, world, ms_total), "unit": UNIT,
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "s8 weights x f16 activations, f32 accumulate", "data": "synthetic", "config": cfg,
+    return {
+        "workload": (f"{sh.name} layer, prefill {sh.T} tokens with the two-layers-ahead predictor scored per token; "
+                     f"cache of {n_hot} HOT + {n_stage} STAGE slots for {E} experts, the other experts are staged "
+                     "from pinned host memory every step and run as later waves"),
+        "tokens": sh.T, **st, "tokens_per_s": world * sh.T / (ms_step / 1e3), "gpu_launches": int(launches),
+        "clocks": clock_record(sampler, lo, hi, ms_step), "hot_experts": hot,
         "roofline": {"bound": "tensor", "kernel": "k_ffn_tc<up/gate>, summed over the waves of a step",
-                     "achieved": ach, "peak": tflops, "unit": "TFLOP/s", "frac": (ach / tflops) if ach else None,
+                     "achieved": ach, "peak": tf_sus, "unit": "TFLOP/s", "frac": (ach / tf_sus) if ach else None,
+                     "frac_of_burst_peak": (ach / tf_burst) if ach else None,
+                     "frac_of_nominal_2250TFLOPs": (ach / NOMINAL_TFLOPS) if ach else None,
                      "peak_source": src + " (cuBLAS bf16, sustained)", "traffic": None,
                      "kernel_ms_per_step": {k: round(v[0] / n_prof, 4) for k, v in prof.items()}},
         "staging": {"bytes_per_step": bytes_staged, "experts_per_step": bytes_staged / m.expert_bytes,
@@ -659,25 +726,15 @@ def run_staged(args):
         "scale_only_staging": {"shared_scale_us_per_expert": scale_shared_us, "per_matrix_scales_us_per_expert": scale_three_us,
                                "ratio": scale_three_us / scale_shared_us,
                                "note": "one bf16[R] copy against three copies (bf16[R], bf16[R], bf16[C]) from pinned host memory"},
-        "e2e": {"value": replica_throughput(sh.T, args.steps, world, ms_total), "unit": UNIT,
+        "e2e": {"value": world * sh.T / (ms_step / 1e3), "unit": UNIT,
                 "h2d_bytes_per_step": int(bytes_staged), "d2h_bytes_per_step": E * 4,
                 "note": "hidden states resident; the staged experts and the counts cross PCIe inside the timed region"},
-        "gpu_launches": int(launches), "clocks": clocks,
     }
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
 
 
-def run_stack(args):
-    """The fifth workload: a 24-layer stack of the fine-grained layer decoded with beam search of width 4; per layer
-    a cache of 12 HOT + 3 STAGE slots for the 60 routed experts (25 %) plus the 4 shared experts, predictor-driven
-    and on-demand staging from pinned host memory on a side stream. One bench step = one decode step (24 layer
-    steps of 4 tokens each plus the harness glue: norm, output head, beam step)."""
+def _single_workload_setup():
     import torch
     import torch.distributed as dist
-    from paper_2609_38090_b200.stack import MoEStack, StackConfig
-
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -685,6 +742,51 @@ def run_stack(args):
     torch.cuda.set_device(dev)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.wait_started()
+    return world, rank, dev, barrier, sampler
+
+
+def _print_record(rec, args, world, rank, sampler, config):
+    import torch.distributed as dist
+    if sampler:
+        sampler.stop()
+    if rank == 0:
+        line = {"metric": METRIC, "value": rec["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "s8 weights x f16 activations, f32 accumulate", "data": "synthetic",
+                "config": config}
+        line.update({k: v for k, v in rec.items() if k not in ("tokens_per_s", "ms_per_step")})
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_staged(args):
+    """`--mode staged`: the third workload alone. One GPU; ranks > 0 of a multi-GPU launch run the same step as
+    independent replicas."""
+    world, rank, dev, barrier, sampler = _single_workload_setup()
+    layer = ResidentLayer(shape_of("mixtral", args.tokens or 2048), dev)
+    rec = staged_record(args, layer, sampler, barrier, dev, world, rank)
+    cfg = workload_config(layer.sh)
+    cfg["workload"] = rec["workload"]
+    _print_record(rec, args, world, rank, sampler, cfg)
+
+
+def stack_record(args, sampler, barrier, dev, world, rank, steps):
+    """The fifth workload: a 24-layer stack of the fine-grained layer decoded with beam search of width 4; per layer
+    a cache of 12 HOT + 3 STAGE slots for the 60 routed experts (25 %) plus the 4 shared experts, predictor-driven
+    and on-demand staging from pinned host memory on a side stream. One step = one decode step (24 layer steps of
+    4 tokens each plus the harness glue: norm, output head, beam step). Also timed with every expert resident."""
+    import torch
+    from paper_2609_38090_b200.stack import MoEStack, StackConfig
+
     sh = inputs.FINE_STACK
     n_hot, n_stage, budget = 12, 3, None
     if args.expert_budget_gb:                # byte budget -> slots, as the cache section of the paper describes
@@ -696,67 +798,58 @@ def run_stack(args):
                       native_step=not args.python_steps)
     st = MoEStack(cfg, device=dev)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
+    def stepper(stack, n_warm):
+        """One decode step per call, continuing one beam search (the expert traffic of a search that restarts
+        every step would be the same few experts over and over)."""
+        hist, sc = stack.decode(n_warm)
+        state = [hist[-1], sc]
 
-    sampler = ClockSampler(local) if rank == 0 else None
-    if sampler:
-        sampler.wait_started()
-    st.decode(args.warmup)
+        def fn(i):
+            h, s_ = stack.decode(1, state[0], state[1])
+            state[0], state[1] = h[-1], s_
+        return fn
+    step_fn = stepper(st, max(args.warmup, 3))
     barrier()
     st.reset_stats()
     launches0 = st.m.kernel_launches
     lo = sampler.mark() if sampler else 0
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    st.decode(args.steps)
-    b.record()
-    barrier()
-    ms_total = reduce_max_ms(a.elapsed_time(b), dev, world)
-    launches = st.m.kernel_launches - launches0
+    blocks = timed_blocks(step_fn, steps, barrier, dev, world)
+    hi = sampler.mark() if sampler else 0
+    bs = block_stats(blocks, steps)
+    n_steps = steps * len(blocks)
+    ms_total = sum(blocks)
+    launches = (st.m.kernel_launches - launches0) // len(blocks)
     code, missing = st.m.poll_status()
     assert code == 0, f"device status {code}, missing experts {missing}"
-    clocks = None
-    if sampler:
-        clocks = sampler.summary(lo, max(sampler.mark(), lo + 1))
-        sampler.stop()
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    hbm, tflops, src = peaks()
+    hbm, tf_sus, tf_burst, src = peaks()
     stats = st.stats()
     cov = st.coverage()
     W, L = sh.T, cfg.n_layers
-    ms_step = ms_total / args.steps
-    layer_steps = args.steps * L
+    ms_step = bs["ms_per_step"]
+    layer_steps = n_steps * L
     be = st.m.expert_bytes
     # distinct experts a layer step touches (for the algorithmic bytes): the routed ones from the cache statistics
     # plus the shared ones, which every step uses
     experts_per_layer_step = (stats.experts_hot + stats.experts_stage + stats.experts_demand) / layer_steps + sh.n_shared
     alg_bytes = experts_per_layer_step * be
-    layer_ms = ms_total / layer_steps
-    cfgj = workload_config(sh)
-    cfgj["workload"] = (f"{L}-layer stack of the fine-grained layer (hidden {sh.C}, ffn {sh.R}, {sh.E} experts top-{sh.k} + "
-                        f"{sh.n_shared} shared), beam width {W}, {args.steps} decode steps; per layer {cfg.n_hot} HOT + "
-                        f"{cfg.n_stage} STAGE slots of {sh.E} routed experts, predictor-driven and on-demand staging from pinned host memory")
-    cfgj["layers"] = L
-    line = {
-        "metric": METRIC, "value": world * W * layer_steps / (ms_total / 1e3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "s8 weights x f16 activations, f32 accumulate",
-        "data": "synthetic", "config": cfgj,
-        "beam_tokens_per_s": world * W * args.steps / (ms_total / 1e3),
+    layer_ms = ms_step / L
+    bytes_staged, copies = st.bytes_staged, stats.copies
+    rec = {
+        "workload": (f"{L}-layer stack of the fine-grained layer (hidden {sh.C}, ffn {sh.R}, {sh.E} experts top-{sh.k} + "
+                     f"{sh.n_shared} shared), beam width {W}, {steps} decode steps per block; per layer {cfg.n_hot} HOT + "
+                     f"{cfg.n_stage} STAGE slots of {sh.E} routed experts, predictor-driven and on-demand staging from pinned host memory"),
+        "tokens": W, "layers": L, **bs, "tokens_per_s": world * W * L / (ms_step / 1e3),
+        "beam_tokens_per_s": world * W / (ms_step / 1e3), "gpu_launches": int(launches),
+        "clocks": clock_record(sampler, lo, hi, ms_step),
         "roofline": {"bound": "hbm", "kernel": "whole layer step (route, predictor, waves of up/gate + down, combine, host read-back)",
                      "achieved": alg_bytes / (layer_ms / 1e3) / 1e9, "peak": hbm, "unit": "GB/s",
-                     "frac": alg_bytes / (layer_ms / 1e3) / 1e9 / hbm, "peak_source": src, "traffic": None,
+                     "frac": alg_bytes / (layer_ms / 1e3) / 1e9 / hbm,
+                     "frac_of_nominal_8TBps": alg_bytes / (layer_ms / 1e3) / 1e9 / NOMINAL_HBM_GBS, "peak_source": src, "traffic": None,
                      "algorithmic_bytes_per_layer_step": alg_bytes, "us_per_layer_step": 1e3 * layer_ms,
                      "note": "latency bound: 4 tokens per layer step; the host-side cache manager reads the routing counts of every layer (a flag in host-mapped memory with the library runtime, a stream synchronisation with --python-steps)",
                      "layer_step": "mira_stack_layer_step (library runtime)" if st.native is not None else "issued from Python call by call"},
         "cache": {"shares_of_routed_pairs": stats.shares(), "experts_per_layer_step": experts_per_layer_step,
-                  "copies_per_decode_step": stats.copies / args.steps, "h2d_bytes_per_decode_step": st.bytes_staged / args.steps,
+                  "copies_per_decode_step": copies / n_steps, "h2d_bytes_per_decode_step": bytes_staged / n_steps,
                   "budget": None if budget is None else {"expert_bytes_gb": args.expert_budget_gb, "mode": budget.mode,
                                                           "n_hot": budget.n_hot, "n_stage": budget.n_stage,
                                                           "share_of_routed_experts_in_slots": budget.slots_per_layer / sh.E},
@@ -765,14 +858,32 @@ def run_stack(args):
                   "hot_swaps": st.hot_swaps(),
                   "prefetch": {"issued": stats.prefetch_issued, "useful": stats.prefetch_useful,
                                "declined": stats.prefetch_declined, "skipped": stats.prefetch_skipped}},
-        "e2e": {"value": world * W * layer_steps / (ms_total / 1e3), "unit": UNIT,
-                "h2d_bytes_per_step": int(st.bytes_staged / args.steps), "d2h_bytes_per_step": L * (sh.E + sh.n_shared + cfg.k_pred) * 4,
+        "e2e": {"value": world * W * L / (ms_step / 1e3), "unit": UNIT,
+                "h2d_bytes_per_step": int(bytes_staged / n_steps), "d2h_bytes_per_step": L * (sh.E + sh.n_shared + cfg.k_pred) * 4,
                 "note": "the staged experts and the per-layer counts / predicted ids cross PCIe inside the timed region"},
-        "gpu_launches": int(launches), "clocks": clocks,
     }
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    del st
+    torch.cuda.empty_cache()
+    if not args.expert_budget_gb:
+        # the same stack with every expert resident: what the layer kernels and the runtime cost without copies
+        full = MoEStack(StackConfig(shape=sh, n_layers=24, vocab=1024, n_hot=sh.E, n_stage=1, k_pred=0, seed=1,
+                                    native_step=not args.python_steps), device=dev)
+        fb = block_stats(timed_blocks(stepper(full, max(args.warmup, 3)), steps, barrier, dev, world), steps)
+        rec["all_resident"] = {"ms_per_step": fb["ms_per_step"], "ms_per_step_best": fb["ms_per_step_best"],
+                               "us_per_layer_step": 1e3 * fb["ms_per_step"] / L,
+                               "tokens_per_s": world * W * L / (fb["ms_per_step"] / 1e3)}
+        del full
+        torch.cuda.empty_cache()
+    return rec
+
+
+def run_stack(args):
+    world, rank, dev, barrier, sampler = _single_workload_setup()
+    rec = stack_record(args, sampler, barrier, dev, world, rank, steps=args.steps)
+    cfgj = workload_config(inputs.FINE_STACK)
+    cfgj["workload"] = rec["workload"]
+    cfgj["layers"] = 24
+    _print_record(rec, args, world, rank, sampler, cfgj)
 
 
 def main():
@@ -785,6 +896,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--ref-tokens", type=int, default=4, help="tokens of the bounded oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="time the headline configuration only (the default run adds one record per other configuration)")
     ap.add_argument("--k-pred", type=int, default=4, help="stack workload: expert ids requested from each predictor head")
     ap.add_argument("--expert-budget-gb", type=float, default=0.0,
                     help="stack workload: device bytes for expert slots of all layers (default: 12 HOT + 3 STAGE per layer)")

@@ -54,7 +54,8 @@ typedef enum {
     MIRA_ERR_NO_PREDICTOR = 5, /* mira_predict on one of the last two layers                  */
     MIRA_ERR_WORKSPACE = 6,    /* workspace too small or T > max_tokens                       */
     MIRA_ERR_CUDA = 7,         /* a CUDA runtime call or a kernel launch failed               */
-    MIRA_ERR_UNSUPPORTED = 8
+    MIRA_ERR_UNSUPPORTED = 8,
+    MIRA_ERR_TIMEOUT = 9       /* (poll) a bounded wait inside a tensor-core kernel ran out; that step's output is undefined */
 } mira_status;
 
 typedef struct {
@@ -128,7 +129,7 @@ mira_status mira_stage_expert(mira_ctx* ctx, const void* pinned_host_blob, void*
 
 /* Section IV-E, linear head on the hidden state: scores the experts of layer `layer + 2`.
  *   token score[t][e] = sum_c hidden[t][c] * pred_w[e][c] + pred_b[e]      (fp32 accumulation)
- *   out_expert_scores[e] = mean over t (summed in token order)
+ *   out_expert_scores[e] = mean over t (fp32; 32 interleaved partial sums over the tokens, added pairwise, divided by T)
  *   out_topk_ids = the k_pred best pooled scores, ties to the lower id.
  * hidden [T][C] bf16, pred_w [E][C] bf16, pred_b [E] fp32 or NULL, out_token_scores [T][E] or NULL,
  * out_topk_ids [k_pred] or NULL (then k_pred is ignored). Heads exist for every layer except the
@@ -201,7 +202,10 @@ mira_status mira_moe_experts(mira_ctx* ctx, const void* hidden, int32_t T,
 
 /* Synchronises `stream`, reads the device status word and clears it. Returns MIRA_OK,
  * MIRA_ERR_EXPERT_MISS (then miss_mask_out, host, ceil((E+n_shared)/32) words or NULL, receives
- * the experts that were needed but not resident) or MIRA_ERR_CUDA. */
+ * the experts that were needed but not resident), MIRA_ERR_TIMEOUT (a pipeline wait of a tensor-core kernel gave
+ * up after its poll limit: every such wait is bounded, the kernel frees its tensor memory and returns, the
+ * outputs of that step are undefined and the context stays usable; reported in preference to a miss, and the
+ * mask is still filled if both happened) or MIRA_ERR_CUDA. */
 mira_status mira_poll_status(mira_ctx* ctx, uint32_t* miss_mask_out, void* stream);
 
 /* Profiling aid. While enabled, every kernel launch made through this context is bracketed by a
@@ -253,12 +257,15 @@ mira_status mira_predict_mixture(mira_ctx* ctx, int32_t layer, const void* hidde
  * mma.sync kernels, also for the batch sizes that would take the tcgen05 kernels (used by the
  * tests to compare the two paths). MIRA_OPT_TENSOR_LAYOUT (value 0..3): 0 lets every step choose the tile layout of
  * the tcgen05 kernels from its token count (the default); 1, 2, 3 force the narrow, wide or big layout, for tests
- * and tuning. MIRA_OPT_UP_CONVERSION (value 0..2): how the up/gate kernels turn int8 codes into fp16 operands. 0 (the
- * default) decides per batch on the device: codes go in as (code + 128) * 2^-24 with the offset taken out afterwards,
- * unless some token's activations have a sum so large against their norm (hidden size * |sum x| > 8192 * |x|_2)
- * that the subtraction would cost accuracy, in which case the codes are converted exactly; 1 forces the exact
- * conversion, 2 the offset form (tests and tuning). */
-enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2, MIRA_OPT_UP_CONVERSION = 3 };
+ * and tuning. MIRA_OPT_UP_CONVERSION (value 0..2): how the tcgen05 up/gate kernel turns int8 codes into fp16 operands
+ * (the weight-streaming kernels always convert exactly). 0 (the default) decides per batch on the device: codes go in
+ * as (code + 128) * 2^-24 with the offset taken out afterwards, unless some token's activations have a sum so large
+ * against their norm (hidden size * |sum x| > 24576 * |x|_2) that the subtraction would cost accuracy, in which case
+ * the codes are converted exactly; 1 forces the exact conversion, 2 the offset form (tests and tuning). MIRA_OPT_TEST_WAIT_TIMEOUT (value 1; test hook): the next tcgen05
+ * up/gate launch of this context leaves out one activation load in its first CTA and gives up its waits after 4096
+ * polls instead of 2^24, so that CTA takes the time-out path (status MIRA_ERR_TIMEOUT at the next poll); the option
+ * clears itself with that launch. */
+enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2, MIRA_OPT_UP_CONVERSION = 3, MIRA_OPT_TEST_WAIT_TIMEOUT = 4 };
 mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value);
 
 /* ---------------------------------------------------------------------------------------------------------------

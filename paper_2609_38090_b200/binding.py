@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmira.so")
 
 MIRA_OK, MIRA_ERR_INVALID_ARG, MIRA_ERR_SHAPE, MIRA_ERR_ALIGN, MIRA_ERR_EXPERT_MISS = 0, 1, 2, 3, 4
-MIRA_ERR_NO_PREDICTOR, MIRA_ERR_WORKSPACE, MIRA_ERR_CUDA, MIRA_ERR_UNSUPPORTED = 5, 6, 7, 8
+MIRA_ERR_NO_PREDICTOR, MIRA_ERR_WORKSPACE, MIRA_ERR_CUDA, MIRA_ERR_UNSUPPORTED, MIRA_ERR_TIMEOUT = 5, 6, 7, 8, 9
 
 
 class mira_config(C.Structure):
@@ -120,6 +120,7 @@ mira_set_option = lib.mira_set_option
 MIRA_OPT_FORCE_DECODE_PATH = 1
 MIRA_OPT_TENSOR_LAYOUT = 2
 MIRA_OPT_UP_CONVERSION = 3
+MIRA_OPT_TEST_WAIT_TIMEOUT = 4
 mira_profile_read = lib.mira_profile_read
 KERNEL_CLASSES = ("route", "group", "schedule", "up_gate", "down", "combine", "scores", "pool", "quantize", "unpack")
 mira_status_string = lib.mira_status_string
@@ -328,7 +329,7 @@ class Mira:
         words = (self.E + self.ns + 31) // 32
         mask = (C.c_uint32 * words)()
         code = mira_poll_status(self._ctx, mask, _stream(stream))
-        missing = [e for e in range(self.E + self.ns) if (mask[e >> 5] >> (e & 31)) & 1] if code == MIRA_ERR_EXPERT_MISS else []
+        missing = [e for e in range(self.E + self.ns) if (mask[e >> 5] >> (e & 31)) & 1] if code in (MIRA_ERR_EXPERT_MISS, MIRA_ERR_TIMEOUT) else []
         return code, missing
 
     def force_decode_path(self, on: bool) -> None:
@@ -341,6 +342,10 @@ class Mira:
     def up_conversion(self, mode: int) -> None:
         """0: decided per batch on the device (default); 1: exact code conversion in the up/gate kernels; 2: offset subnormals."""
         _check(mira_set_option(self._ctx, MIRA_OPT_UP_CONVERSION, int(mode)), "mira_set_option")
+
+    def test_wait_timeout(self) -> None:
+        """Test hook: the next tcgen05 up/gate launch takes its time-out path in one CTA (see MIRA_OPT_TEST_WAIT_TIMEOUT)."""
+        _check(mira_set_option(self._ctx, MIRA_OPT_TEST_WAIT_TIMEOUT, 1), "mira_set_option")
 
     def profile(self, enable: bool) -> None:
         _check(mira_profile(self._ctx, int(enable)), "mira_profile")

@@ -348,10 +348,15 @@ mira_status mira_poll_status(mira_ctx* ctx, uint32_t* miss_mask_out, void* strea
     int32_t host[32];
     MIRA_CUDA_OK(cudaMemcpy(host, ctx->ws + ctx->lay.status, sizeof(host), cudaMemcpyDeviceToHost));
     if (host[0] == 0) return MIRA_OK;
+    // status word: bit 0 = a routed expert had no slot (the miss mask says which), bit 1 = a bounded wait of a
+    // tensor-core kernel ran out. The time-out is reported in preference: that step's outputs are undefined.
     const int words = (Et(ctx->cfg) + 31) / 32;
-    if (miss_mask_out) std::memcpy(miss_mask_out, host + 16, (size_t)words * 4);
+    if (miss_mask_out) {
+        if (host[0] & 1) std::memcpy(miss_mask_out, host + 16, (size_t)words * 4);
+        else std::memset(miss_mask_out, 0, (size_t)words * 4);
+    }
     MIRA_CUDA_OK(cudaMemset(ctx->ws + ctx->lay.status, 0, 24 * sizeof(int32_t)));   // status + miss mask, not the done mask
-    return MIRA_ERR_EXPERT_MISS;
+    return (host[0] & 2) ? MIRA_ERR_TIMEOUT : MIRA_ERR_EXPERT_MISS;
 }
 
 mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value) {
@@ -359,6 +364,7 @@ mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value) {
     if (option == MIRA_OPT_FORCE_DECODE_PATH) { ctx->force_decode_path = value != 0; return MIRA_OK; }
     if (option == MIRA_OPT_TENSOR_LAYOUT && value >= 0 && value <= 3) { ctx->tc_layout = value; return MIRA_OK; }
     if (option == MIRA_OPT_UP_CONVERSION && value >= 0 && value <= 2) { ctx->up_conversion = value; return MIRA_OK; }
+    if (option == MIRA_OPT_TEST_WAIT_TIMEOUT) { ctx->test_wait_timeout = value != 0; return MIRA_OK; }
     return MIRA_ERR_INVALID_ARG;
 }
 
@@ -375,6 +381,7 @@ const char* mira_status_string(mira_status s) {
         case MIRA_ERR_WORKSPACE: return "workspace too small";
         case MIRA_ERR_CUDA: return "CUDA error";
         case MIRA_ERR_UNSUPPORTED: return "unsupported";
+        case MIRA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     }
     return "unknown";
 }

@@ -42,20 +42,15 @@ __device__ __forceinline__ void mma16816(float (&c)[4], unsigned a0, unsigned a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Four int8 codes (one 32-bit word, already XOR-ed with 0x80808080 so each byte is u = code + 128)
-// -> two half2 whose bit patterns are 0x00uu: the fp16 SUBNORMAL u * 2^-24, exactly, with no offset to
-// subtract. The MMA therefore accumulates 2^-24 * sum_k (code_k + 128) b_k; the epilogue multiplies by
-// 2^24 and subtracts 128 * sum_k b_k (the column sum of the activation tile, known exactly enough:
-// the cancellation is only ~4x the result, far from fp32 trouble). Three ALU operations per four
-// weights (one XOR, two byte permutes).
-__device__ __forceinline__ unsigned cvt_lo(unsigned u) { return __byte_perm(u, 0u, 0x4140); }
-__device__ __forceinline__ unsigned cvt_hi(unsigned u) { return __byte_perm(u, 0u, 0x4342); }
-constexpr float kTwo24 = 16777216.f;
-// Exact alternative: the byte goes into the mantissa of 1024.0 (0x6400 | u = 1024 + u) and 1152 = 1024 + 128 is
-// subtracted, which leaves the signed code itself. Two more half2 subtractions per four weights, no offset to undo.
-// The down kernel uses it: its offset term would need the column sums of the fp16 intermediate, one extra MMA per
-// two weight MMAs (measured: 94.6 -> 88.7 us at 8 tokens per expert, 163 -> 137 us at 32). The up/gate kernel
-// keeps the subnormal form, whose offset term is the per-token sum the routing kernel already has.
+// Four int8 codes (one 32-bit word, already XOR-ed with 0x80808080 so each byte is u = code + 128) -> two half2 of
+// the signed codes, exactly: the byte goes into the mantissa of 1024.0 (0x6400 | u = 1024 + u) and 1152 = 1024 + 128
+// is subtracted. Five ALU operations per four weights (one XOR, two byte permutes, two half2 subtractions).
+// (Feeding u * 2^-24 as an fp16 subnormal and subtracting 128 * sum(x) afterwards saves the two subtractions, but
+// the tensor cores add in fp32 with truncation, so the subtracted term costs accuracy as soon as a token's
+// activations have a mean: measured 6e-3 instead of 1e-3 at hidden size 4096 with mean = spread. It also needs the
+// token sums in the epilogue. Measured on the Mixtral shape the exact form is as fast at 1 and 8 tokens and 0.5 %
+// slower at 32, so the streaming kernels always convert exactly; the tcgen05 up/gate kernel, where the conversion
+// is on the critical path, keeps the offset form for batches without such a token.)
 __device__ __forceinline__ unsigned cvt_exact_lo(unsigned u) {
     unsigned v = __byte_perm(u, 0x64646464u, 0x4140);
     __half2 r = __hsub2(*reinterpret_cast<__half2*>(&v), __half2half2(__ushort_as_half(0x6480)));
@@ -72,14 +67,14 @@ __device__ __forceinline__ float pow2i(int e) { return __uint_as_float((unsigned
 __device__ __forceinline__ int expo(float v) { return (int)((__float_as_uint(v) >> 23) & 0xff) - 127; }
 
 struct ItemTable {             // the schedule, copied to shared memory once per CTA
-    int n_active, total_tb, dc_heavy;
+    int n_active, total_tb;
     int tb_prefix[kMaxExperts + 1];
     int w_prefix[kMaxExperts + 1];     // cost prefix of this kernel (up/gate or down)
     uint8_t act_expert[kMaxExperts];
 };
 
 __device__ __forceinline__ void load_table(ItemTable& tab, const Sched* __restrict__ sched, int which) {
-    if (threadIdx.x == 0) { tab.n_active = sched->n_active; tab.total_tb = sched->total_tb; tab.dc_heavy = sched->dc_heavy; }
+    if (threadIdx.x == 0) { tab.n_active = sched->n_active; tab.total_tb = sched->total_tb; }
     for (int i = threadIdx.x; i < kMaxExperts; i += blockDim.x) tab.act_expert[i] = (uint8_t)sched->act_expert[i];
     for (int i = threadIdx.x; i <= kMaxExperts; i += blockDim.x) {
         tab.tb_prefix[i] = sched->tb_prefix[i];
@@ -121,7 +116,6 @@ struct FfnArgs {
     const int32_t* row_token;
     const float* xscale;
     const float* xnorm;
-    const float* xsum;          // sum over c of the fp16 (pre-scaled) activations of each token
     const int32_t* hexp;        // per expert: exponent of the intermediate's expected magnitude per unit of |x|^2
     float* hscale;
     const __half* x16;
@@ -130,7 +124,6 @@ struct FfnArgs {
     int R, C, act_on_w1;
     int down_splits, down_slice;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
-    int up_conversion;          // up/gate codes: 0 as the schedule's dc_heavy flag says, 1 exact, 2 offset subnormals
     long ypart_stride;          // elements between two splits = P * C
 };
 
@@ -287,7 +280,7 @@ __device__ __forceinline__ void start_step_acts(CopyState& c, const StepDesc& d)
 
 // Runs one step whose first stages are already in flight (start_step), then starts the next step's first
 // stages before its own epilogue, so the memory system never idles between steps.
-template <bool DOWN, int NT, bool EXACT>
+template <bool DOWN, int NT>
 __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, CopyState& cs, const StepDesc& next,
                                          CopyState& cs_next, unsigned char* ringA) {
     constexpr int kStages = stages_for(NT);
@@ -336,8 +329,7 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
             for (int j = 0; j < 4; ++j) {
                 const unsigned ua = wa[j] ^ 0x80808080u, ub = wb[j] ^ 0x80808080u;
                 unsigned f0, f1, f2, f3;
-                if (EXACT) { f0 = cvt_exact_lo(ua); f2 = cvt_exact_hi(ua); f1 = cvt_exact_lo(ub); f3 = cvt_exact_hi(ub); }
-                else { f0 = cvt_lo(ua); f2 = cvt_hi(ua); f1 = cvt_lo(ub); f3 = cvt_hi(ub); }
+                f0 = cvt_exact_lo(ua); f2 = cvt_exact_hi(ua); f1 = cvt_exact_lo(ub); f3 = cvt_exact_hi(ub);
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) mma16816(acc[mt][nt], f0, f1, f2, f3, bf[nt][2 * j], bf[nt][2 * j + 1]);
             }
@@ -368,20 +360,6 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
     const bool early = next.valid && next.nt == NT;
     if (early) cs_next = start_step<DOWN>(A, next, sA);
 
-    // undo the 2^-24 of the subnormal weights and the +128 offset: acc <- 2^24 acc - 128 * column sum
-    if (active && !EXACT) {
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const float colsum = half ? 0.f : A.xsum[A.row_token[pos0 + min(nt * 8 + tq * 2 + i, ntok - 1)]];   // whole-row sum: count it once
-#pragma unroll
-                for (int mt = 0; mt < kMT; ++mt) {
-                    acc[mt][nt][i] = fmaf(acc[mt][nt][i], kTwo24, -128.f * colsum);
-                    acc[mt][nt][2 + i] = fmaf(acc[mt][nt][2 + i], kTwo24, -128.f * colsum);
-                }
-            }
-    }
     // Add the two halves of the reduction in two passes through the pair's exchange slot: warp `half` keeps
     // m-tile `half` and receives the other warp's partial sums of that m-tile; always (warp 0 part) + (warp 1 part).
     float* slot = reinterpret_cast<float*>(ringA + ring_bytes(NT)) + (size_t)pair * 128 * NT;
@@ -495,7 +473,6 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     long u = unit_at(tab, cost * blockIdx.x / gridDim.x, per_tb, w_full);
     const long u1 = unit_at(tab, cost * (blockIdx.x + 1) / gridDim.x, per_tb, w_full);
     const unsigned sA = (unsigned)__cvta_generic_to_shared(ringA);
-    const bool exact_up = A.up_conversion == 1 || (A.up_conversion == 0 && tab.dc_heavy != 0);
 
     // Describes the step that starts at unit v (valid = false past the end of this CTA's range).
     auto decode = [&](long v) {
@@ -540,20 +517,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         u += cur.nstep;
         const StepDesc next = decode(u);
         CopyState cs_next = cs;
-        if (DOWN || exact_up) {
-            switch (cur.nt) {
-                case 1: ffn_step<DOWN, 1, true>(A, cur, cs, next, cs_next, ringA); break;
-                case 2: ffn_step<DOWN, 2, true>(A, cur, cs, next, cs_next, ringA); break;
-                case 3: ffn_step<DOWN, 3, true>(A, cur, cs, next, cs_next, ringA); break;
-                default: ffn_step<DOWN, 4, true>(A, cur, cs, next, cs_next, ringA); break;
-            }
-        } else {
-            switch (cur.nt) {
-                case 1: ffn_step<false, 1, false>(A, cur, cs, next, cs_next, ringA); break;
-                case 2: ffn_step<false, 2, false>(A, cur, cs, next, cs_next, ringA); break;
-                case 3: ffn_step<false, 3, false>(A, cur, cs, next, cs_next, ringA); break;
-                default: ffn_step<false, 4, false>(A, cur, cs, next, cs_next, ringA); break;
-            }
+        switch (cur.nt) {
+            case 1: ffn_step<DOWN, 1>(A, cur, cs, next, cs_next, ringA); break;
+            case 2: ffn_step<DOWN, 2>(A, cur, cs, next, cs_next, ringA); break;
+            case 3: ffn_step<DOWN, 3>(A, cur, cs, next, cs_next, ringA); break;
+            default: ffn_step<DOWN, 4>(A, cur, cs, next, cs_next, ringA); break;
         }
         cur = next;
         cs = cs_next;
@@ -655,10 +623,8 @@ FfnArgs make_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) {
     A.row_token = ws_ptr<int32_t>(ctx, ctx->lay.row_token);
     A.xscale = ws_ptr<float>(ctx, ctx->lay.xscale);
     A.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm);
-    A.xsum = ws_ptr<float>(ctx, ctx->lay.xsum);
     A.hscale = ws_ptr<float>(ctx, ctx->lay.hscale);
     A.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
-    A.up_conversion = ctx->up_conversion;
     A.x16 = ws_ptr<__half>(ctx, ctx->lay.x16);
     A.h16 = ws_ptr<__half>(ctx, ctx->lay.h16);
     A.ypart = ws_ptr<float>(ctx, ctx->lay.ypart);

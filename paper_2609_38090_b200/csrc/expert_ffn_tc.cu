@@ -90,6 +90,9 @@ struct TcArgs {
     int R, C, act_on_w1;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
     int up_conversion;          // up/gate codes: 0 as the schedule's dc_heavy flag says, 1 exact, 2 offset subnormals
+    uint32_t spin_limit;        // polls after which a barrier wait gives up (kSpinLimit; shortened by MIRA_OPT_TEST_WAIT_TIMEOUT)
+    int drop_first_load;        // test hook: CTA 0 leaves out the activation load of its first K-block, so the waits on that
+                                // stage run out and the kernel leaves through its time-out path
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -113,8 +116,8 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {      
     return ok != 0;
 }
 // Bounded wait. Returns false (and raises the abort flag) if the barrier did not flip in time.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_try(bar, parity)) return true;
         if ((spin & 1023u) == 1023u && *abort_flag) return false;
     }
@@ -343,7 +346,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 }
                 const uint32_t g = gbase + (uint32_t)(kb0 + kGroups * j);
                 const uint32_t st = g % kAStages;
-                if (!mbar_wait(a_empty(st), ((g / kAStages) & 1u) ^ 1u, &s_abort)) { ok = false; break; }
+                if (!mbar_wait(a_empty(st), ((g / kAStages) & 1u) ^ 1u, &s_abort, A.spin_limit)) { ok = false; break; }
                 tc_fence_after();
                 __syncwarp();
                 tmem_st32(tmem + ((uint32_t)(gw * 32) << 16) + kTmemA + st * 32, f);   // TMEM lane = MMA row
@@ -363,7 +366,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
         for (long tile = blockIdx.x; tile < total && !s_abort; tile += gridDim.x, ++it) {
             const Tile t = decode(tile);
             const int buf = (int)(it % kAccBufs);
-            if (!mbar_wait(acc_full(buf), (uint32_t)((it / kAccBufs) & 1), &s_abort)) break;
+            if (!mbar_wait(acc_full(buf), (uint32_t)((it / kAccBufs) & 1), &s_abort, A.spin_limit)) break;
             tc_fence_after();
             const uint32_t acc_t = lane_base + buf * kTileN;
             const int ncol = (t.ntok + 31) & ~31;
@@ -429,7 +432,11 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 const uint32_t box_bytes = (uint32_t)(hi + 1) * kBoxStep * kKB * 2;
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait(b_empty(st), ph, &s_abort)) { ok = false; break; }
+                    if (!mbar_wait(b_empty(st), ph, &s_abort, A.spin_limit)) { ok = false; break; }
+                    if (A.drop_first_load && blockIdx.x == 0 && tile == blockIdx.x && kb == 0) {    // test hook, see TcArgs
+                        if (++st == kBStages) { st = 0; ph ^= 1u; }
+                        continue;
+                    }
                     const uint32_t dst = b_s + st * kBTileBytes, bar = b_full(st);
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(box_bytes) : "memory");
                     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
@@ -453,17 +460,17 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
             for (long tile = blockIdx.x; tile < total && !s_abort; tile += gridDim.x) {
                 const Tile t = decode(tile);
                 const uint32_t idesc = make_idesc((t.ntok + 15) & ~15);
-                if (!mbar_wait(acc_empty(buf), pacc, &s_abort)) break;   // its previous epilogue is done
+                if (!mbar_wait(acc_empty(buf), pacc, &s_abort, A.spin_limit)) break;   // its previous epilogue is done
                 tc_fence_after();
                 const uint32_t d_t = tmem + buf * kTileN;
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb, ++g) {
                     if (kIssuers == 2 && (int)(g & 1u) != q) continue;
                     const uint32_t sa = g % kAStages, pa = (g / kAStages) & 1u;
-                    if (!ready && !mbar_wait(a_full(sa), pa, &s_abort)) { ok = false; break; }
+                    if (!ready && !mbar_wait(a_full(sa), pa, &s_abort, A.spin_limit)) { ok = false; break; }
                     if (kIssuers == 2 && g > 0) {            // the other issuer has issued K-block g - 1
                         const uint32_t n_other = (q == 0) ? nmine - 1 : nmine;      // its blocks before this one, minus one
-                        if (!mbar_wait(turn(q), n_other & 1u, &s_abort)) { ok = false; break; }
+                        if (!mbar_wait(turn(q), n_other & 1u, &s_abort, A.spin_limit)) { ok = false; break; }
                     }
                     tc_fence_after();
                     const uint32_t a_t = tmem + kTmemA + sa * 32;
@@ -487,9 +494,9 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
         }
     }
     // ---------------------------------------------------- common exit
-    if (s_abort && tid == 0) atomicOr(A.status, 2);
     tc_fence_before();
     __syncthreads();
+    if (s_abort && tid == 0) atomicOr(A.status, 2);      // after the barrier: the role that gave up may be the last to arrive
     if (warp == kTmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -559,6 +566,8 @@ TcArgs make_tc_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) 
     A.R = ctx->cfg.ffn; A.C = ctx->cfg.hidden; A.act_on_w1 = ctx->cfg.act_on_w1;
     A.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX;
     A.up_conversion = ctx->up_conversion;
+    A.spin_limit = kSpinLimit;
+    A.drop_first_load = 0;
     return A;
 }
 
@@ -634,6 +643,11 @@ mira_status launch_up_gate_tc(mira_ctx* ctx, void* const* slots, const int32_t* 
     G.sum_pos = ws_ptr<float>(ctx, ctx->lay.sum_pos); G.xsum = ws_ptr<float>(ctx, ctx->lay.xsum);
     G.hscale = ws_ptr<float>(ctx, ctx->lay.hscale); G.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
     G.C = ctx->cfg.hidden; G.R = ctx->cfg.ffn; G.Etot = Et(ctx->cfg);
+    if (ctx->test_wait_timeout) {          // one launch whose waits run out (MIRA_OPT_TEST_WAIT_TIMEOUT)
+        A.spin_limit = 1u << 12;
+        A.drop_first_load = 1;
+        ctx->test_wait_timeout = false;
+    }
     ProfScope ps(ctx, MIRA_K_UP_GATE, st);
     const int P = ctx->route_T * (ctx->route_k + ctx->cfg.n_shared);
     MIRA_CUDA_OK(launch_pdl(k_gather_x16p, dim3(P), dim3(128), 0, st, G));

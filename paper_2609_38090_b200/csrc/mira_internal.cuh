@@ -102,6 +102,7 @@ struct mira_ctx {
     bool tensor_path_ok = false;
     bool force_decode_path = false;
     int tc_layout = 0;                 // 0: chosen per step; 1..3 force a tile layout of the tensor-core kernels (MIRA_OPT_TENSOR_LAYOUT)
+    bool test_wait_timeout = false;    // the next tcgen05 up/gate launch drops one load and shortens its waits (MIRA_OPT_TEST_WAIT_TIMEOUT)
     int up_conversion = 0;             // 0: chosen per batch on the device; 1: exact; 2: offset subnormals (MIRA_OPT_UP_CONVERSION)
     bool prof_on = false;
     size_t prof_used = 0;

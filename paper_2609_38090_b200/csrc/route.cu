@@ -346,11 +346,12 @@ struct SchedArgs {
     int T, R, C, per_matrix, n_main;    // n_main: CTAs of the launch that are not statistics CTAs
 };
 
-// The up/gate kernels may feed the codes as (code + 128) * 2^-24 and subtract 128 * sum(x) afterwards. The tensor
+// The tcgen05 up/gate kernel may feed the codes as (code + 128) * 2^-24 and subtract 128 * sum(x) afterwards. The tensor
 // cores add in fp32 with truncation, so the subtracted term costs about C / 16 accumulation steps of 2^-24 of ITS
 // size, while the wanted sum is about 32 |x|_2 (codes have an rms near 32): the relative error grows like
-// kappa * C * |sum x| / |x|_2 * 2^-27. A batch takes the exact conversion when any of its tokens exceeds the bound
-// below; zero-mean activations (|sum x| ~ |x|_2) stay under it up to a hidden size of 8192.
+// C * |sum x| / |x|_2 (measured on B200: nothing visible at 11 k, 2e-3 added at 82 k). A batch takes the exact
+// conversion when any of its tokens exceeds the bound below; zero-mean activations (|sum x| a few times |x|_2 at
+// most) stay under it up to a hidden size of about 6000.
 constexpr float kDcBound = 24576.f;     // C * |sum x| / |x|_2 from which the exact conversion is used
 
 // Called by every thread of the CTA that writes the schedule. xsum / xnorm may have been written by other CTAs of

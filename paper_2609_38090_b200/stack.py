@@ -244,11 +244,12 @@ class MoEStack:
         library, the same arithmetic as `rms_norm(x.float() + out.float()).to(bf16)`)."""
         return binding.residual_rmsnorm(x, out, eps=1e-6, stream=self.main)
 
-    def decode(self, n_steps: int, first_tokens=None):
-        """Beam search of width W for n_steps steps. Returns (tokens [n_steps, W], beam scores [W])."""
+    def decode(self, n_steps: int, first_tokens=None, first_scores=None):
+        """Beam search of width W for n_steps steps. Returns (tokens [n_steps, W], beam scores [W]). A search is
+        continued by passing the last row of tokens and the scores of the previous call."""
         W, V = self.W, self.cfg.vocab
         tokens = torch.arange(W, device=self.dev) if first_tokens is None else first_tokens.to(self.dev)
-        scores = torch.zeros(W, dtype=torch.float32, device=self.dev)
+        scores = torch.zeros(W, dtype=torch.float32, device=self.dev) if first_scores is None else first_scores.to(self.dev)
         history = []
         for step in range(n_steps):
             x = self.emb[tokens].contiguous()

@@ -121,3 +121,67 @@ def test_mixtral_shape_in_the_per_matrix_scale_format():
         assert np.array_equal(got[e], ref), f"expert {e}"
     lay.check(8)
     lay.check(256, sample=6)
+
+
+def test_mixtral_prefill_with_predictor_and_a_cache_of_four_hot_and_two_stage_slots(mixtral):
+    """The third workload at its full size: 2048 tokens of the Mixtral-shaped layer, the two-layers-ahead head
+    (hidden 4096 -> 8 scores, top-2) scored per token, and an expert cache of 4 HOT + 2 STAGE slots for the 8
+    experts: the HOT experts run as the first wave while the others are copied from pinned host memory and run
+    as later waves of two. Predictor: per-token scores, pooled scores and ids against the oracle. Layer: sampled
+    rows against the oracle, and the whole output bit for bit against the all-resident call."""
+    sh, m, b = mixtral.sh, mixtral.m, mixtral.b
+    T, n_hot, n_stage = 2048, 4, 2
+    x = inputs.hidden(sh, T, step=1)
+    xd = to_bf16_cuda(x)
+    wp, bp = inputs.predictor(sh)
+    pooled, ts, ids = m.predict(0, xd, to_bf16_cuda(wp), torch.from_numpy(bp).cuda(), k_pred=2, token_scores=True)
+    ts_ref, pooled_ref, ids_ref, margin = oracle.predict(x, wp, bp, k_pred=2)
+    assert np.abs(ts.cpu().numpy() - ts_ref).max() < 1e-4 and np.abs(pooled.cpu().numpy() - pooled_ref).max() < 1e-4
+    assert margin > 1e-4 and np.array_equal(ids.cpu().numpy(), ids_ref)
+
+    resident = m.moe_layer(xd, mixtral.wr_d, mixtral.bias_d, mixtral.slots, mixtral.slot_map, sh.k).clone()
+    r = m.route(xd, mixtral.wr_d, mixtral.bias_d, sh.k)
+    cnt = r["count"].cpu().tolist()
+    hot = sorted(np.argsort(-np.array(cnt), kind="stable")[:n_hot].tolist())
+    cold = [e for e in range(sh.E) if e not in hot and cnt[e] > 0]
+    assert len(cold) == sh.E - n_hot                                  # 2048 tokens reach every expert: two staged waves
+    host = mixtral.blobs_gpu.cpu().pin_memory()
+    cache = torch.zeros((n_hot + n_stage, m.expert_bytes), dtype=torch.uint8, device="cuda")
+    for i, e in enumerate(hot):
+        cache[i].copy_(mixtral.blobs_gpu[e])
+    cslots = b.slot_table(cache)
+
+    def smap(pairs):
+        t = torch.full((sh.E,), -1, dtype=torch.int32)
+        for e, sl in pairs:
+            t[e] = sl
+        return t.cuda()
+    side, main = torch.cuda.Stream(), torch.cuda.current_stream()
+    ready = [torch.cuda.Event() for _ in range(n_stage)]
+    waves = [cold[j:j + n_stage] for j in range(0, len(cold), n_stage)]
+    torch.cuda.synchronize()
+    for sl, e in enumerate(waves[0]):                                 # staged while the HOT wave computes
+        m.stage_expert(host[e], cache[n_hot + sl], side, ready[sl])
+    m.moe_experts(xd, cslots, smap([(e, i) for i, e in enumerate(hot)]), expert_ids=hot, final_wave=False)
+    out = None
+    for wi, wave in enumerate(waves):
+        for sl in range(len(wave)):
+            main.wait_event(ready[sl])
+        out = m.moe_experts(xd, cslots, smap([(e, n_hot + sl) for sl, e in enumerate(wave)]), expert_ids=wave,
+                            final_wave=wi == len(waves) - 1)
+        if wi + 1 < len(waves):
+            done = torch.cuda.Event()
+            done.record(main)
+            side.wait_event(done)                                     # the STAGE slots are free once this wave has run
+            for sl, e in enumerate(waves[wi + 1]):
+                m.stage_expert(host[e], cache[n_hot + sl], side, ready[sl])
+    torch.cuda.synchronize()
+    assert m.poll_status()[0] == 0
+    assert torch.equal(out.view(torch.int16), resident.view(torch.int16))
+    logits = oracle.linear_scores(x, mixtral.wr, mixtral.bias)
+    _, _, _, mrg = oracle.topk_softmax(logits, sh.k)
+    safe = mrg > 1e-5 * np.maximum(1.0, np.abs(logits).max(1))
+    rows = np.array([t for t in np.random.default_rng(9).choice(T, 10, replace=False) if safe[t]])
+    ref = np.stack([oracle.moe_layer(x[t:t + 1], mixtral.wr, mixtral.bias, mixtral.blobs, sh.R, sh.k)["out64"][0] for t in rows])
+    got = out.float().cpu().numpy()[rows]
+    assert gate_b(got, ref) <= TOL and gate_c(got, ref, bf16_output=True) <= TOL

@@ -1,6 +1,6 @@
 """GPU parity on inputs that stress the numerical decisions of the expert kernels rather than their indexing:
-activations with a large mean (the up/gate kernels' offset-subnormal code conversion subtracts 128 * sum(x), which
-must not be used when that sum is large against the norm), and expert weights whose row scales spread over orders
+activations with a large mean (the tcgen05 up/gate kernel's offset-subnormal code conversion subtracts
+128 * sum(x), which must not be used when that sum is large against the norm), and expert weights whose row scales spread over orders
 of magnitude (the fp16 intermediate of the down projection is placed by the expert's largest row scale). The bar is
 the same as everywhere: 2e-3 in the pre-rounding measure, against the oracle, through both kernel families."""
 import numpy as np
@@ -49,7 +49,8 @@ def test_activations_with_a_large_mean(C, mu, T):
     out_bf16 = _run(wl, sh, T, fp32=False).float().cpu().numpy()
     assert gate_b(out_bf16, res["out64"]) <= TOL and gate_c(out_bf16, res["out64"], bf16_output=True) <= TOL
     if C >= 4096:
-        # the decision is taken on the device: such a batch must have run the exact conversion ...
+        # the decision is taken on the device: such a batch must have run the exact conversion ... (the
+        # weight-streaming kernels of the 8-token batch always do)
         assert torch.equal(out, _run(wl, sh, T, conversion=1))
 
 

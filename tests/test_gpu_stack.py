@@ -123,3 +123,38 @@ def test_residual_rmsnorm_glue_matches_the_torch_formula(C):
     assert torch.isfinite(got).all()
     assert ((got - ref).abs() <= ref.abs() * 2.0 ** -7 + 1e-30).all()          # within one bf16 ulp of the fp32 result
     assert ((got - ref.to(torch.bfloat16).float()) != 0).float().mean() < 0.01  # and almost always the same rounding
+
+
+def test_full_size_stack_of_24_fine_grained_layers_teacher_forced():
+    """The fifth workload at its full size: 24 layers of the fine-grained layer (hidden 2048, ffn 1408, 60 experts
+    top-4 plus 4 shared), beam width 4, per layer a cache of 12 HOT + 3 STAGE slots (25 % of the routed experts),
+    predictor-driven and on-demand staging from 13 GB of pinned host memory through the library's layer-step
+    runtime. A few decode steps; sampled (step, layer) calls are recomputed by the oracle from the recorded
+    inputs, with the experts those tokens need compressed by the oracle from the same seeded weights."""
+    from paper_2609_38090_b200.stack import MoEStack, StackConfig
+    sh = inputs.FINE_STACK
+    cfg = StackConfig(shape=sh, n_layers=24, vocab=1024, n_hot=12, n_stage=3, k_pred=4, seed=1)
+    rec = []
+    st = MoEStack(cfg, build="numpy", record=lambda s, l, x, o: rec.append((s, l, x.clone(), o.clone())))
+    tokens, scores = st.decode(3)
+    torch.cuda.synchronize()
+    assert st.m.poll_status()[0] == 0
+    assert tokens.shape == (3, sh.T) and torch.isfinite(scores).all() and len(rec) == 3 * cfg.n_layers
+    stats = st.stats()
+    assert stats.pairs_hot > 0 and stats.pairs_demand > 0 and stats.copies > 0      # the cache was exercised
+    picks = [(0, 0), (0, 11), (0, 23), (1, 5), (1, 22), (2, 1), (2, 17), (2, 23)]
+    for s, l, x, out in (r for r in rec if (r[0], r[1]) in picks):
+        lsh = dataclasses.replace(sh, layer=l, seed=cfg.seed)
+        wr, bias = inputs.router(lsh)
+        xin = x.float().cpu().numpy()
+        logits = oracle.linear_scores(xin, wr, bias)
+        idx, _, _, margin = oracle.topk_softmax(logits, sh.k)
+        if not (margin > 1e-5 * np.maximum(1.0, np.abs(logits).max(1))).all():
+            continue                                                        # a near-tie: either neighbour is a valid routing
+        need = set(idx.ravel().tolist()) | set(range(sh.E, sh.E + sh.n_shared))
+        blobs = [oracle.quantize_expert(*inputs.expert_weights(lsh, e)) if e in need else None
+                 for e in range(sh.E + sh.n_shared)]
+        res = oracle.moe_layer(xin, wr, bias, blobs, sh.R, sh.k, n_shared=sh.n_shared)
+        got = out.float().cpu().numpy()
+        b_, c_ = gate_b(got, res["out64"]), gate_c(got, res["out64"], bf16_output=True)
+        assert b_ <= TOL and c_ <= TOL, f"step {s} layer {l}: gate B {b_}, gate C {c_}"
