@@ -41,13 +41,14 @@ Layout make_layout(const mira_config& c) {
     L.xnorm = o;     o = align256(o + T * 4);
     L.xsum = o;      o = align256(o + T * 4);
     L.hscale = o;    o = align256(o + P * 4);
-    L.hexp = o;      o = align256(o + Etot * 4);
+    L.hexp = o;      o = align256(o + 2 * kMaxExperts * 4);
     L.x16 = o;       o = align256(o + T * C * 2);
     L.x16p = o;      o = align256(o + (T >= (size_t)kTensorPathMinTokens ? P * C * 2 : 0));
     L.xs_pos = o;    o = align256(o + (T >= (size_t)kTensorPathMinTokens ? P * 4 : 0));
     L.hm_pos = o;    o = align256(o + (T >= (size_t)kTensorPathMinTokens ? P * 4 : 0));
     L.sum_pos = o;   o = align256(o + (T >= (size_t)kTensorPathMinTokens ? P * 4 : 0));
     L.h16 = o;       o = align256(o + P * R * 2);
+    L.h16lo = o;     o = align256(o + P * R * 2);
     L.ypart = o;     o = align256(o + std::max(S * P * C * 4, R * 4));   // at least one expert's abs-max scratch for the quantizer
     L.pred = o;      o = align256(o + T * E * 4);
     L.mix = o;       o = align256(o + 8 * (C + E) * 4);

@@ -120,6 +120,7 @@ struct FfnArgs {
     float* hscale;
     const __half* x16;
     __half* h16;
+    __half* h16lo;              // lower window of the intermediate, written and read for wide-range experts only
     float* ypart;
     int R, C, act_on_w1;
     int down_splits, down_slice;
@@ -173,6 +174,8 @@ struct StepDesc {
     const unsigned char* blob;
     int row0, k0, klen, split, pos0, ntok, nt, nstep, hexp;
     bool active, valid;
+    bool wide;          // wide-range expert: the intermediate has a second, lower fp16 window (h16lo)
+    bool last_half;     // S5 of a wide-range expert takes a 32-token block as two halves of 16 (see k_ffn)
 };
 
 // Per-thread state of the copies of one step (geometry follows the step's NT).
@@ -207,11 +210,21 @@ __device__ __forceinline__ CopyState setup_copy(const FfnArgs& A, const StepDesc
     const int bcol = threadIdx.x & 7, btok = threadIdx.x >> 3;
     c.b_tile = d.nt * 8 * kBRow;
     c.b_cp = sA + stages_for(d.nt) * (kPairs * kATile) + btok * kBRow + bcol * 16;
-    c.bvalid = btok < d.ntok;
     {
-        const int tok = min(btok, d.ntok - 1);     // rows beyond ntok alias the last valid row and are not copied
+        // S5 of a wide-range expert: the tile's first nt / 2 n-tiles hold the upper window of the <= 16 tokens, the
+        // other nt / 2 the lower window of the same tokens, so one pass over the weight fragments serves both
+        int trow = btok;
+        const __half* src = DOWN ? A.h16 : A.x16;
+        if (DOWN && d.wide) {
+            const int hr = d.nt * 4;               // rows of one window: 8 * (nt / 2)
+            if (btok >= hr) { trow = btok - hr; src = A.h16lo; }
+            c.bvalid = trow < d.ntok && btok < 2 * hr;
+        } else {
+            c.bvalid = btok < d.ntok;
+        }
+        const int tok = min(trow, d.ntok - 1);     // rows beyond ntok alias the last valid row and are not copied
         const size_t rowi = DOWN ? (size_t)(d.pos0 + tok) : (size_t)A.row_token[d.pos0 + tok];
-        c.b = reinterpret_cast<const unsigned char*>((DOWN ? A.h16 : A.x16) + rowi * ld + d.k0) + bcol * 16;
+        c.b = reinterpret_cast<const unsigned char*>(src + rowi * ld + d.k0) + bcol * 16;
     }
     c.nchunk = d.klen / kChunk;
     c.active = d.active;
@@ -402,6 +415,22 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
             so0 = __bfloat162float(so[row0 + mt * 16 + g]);
             so1 = __bfloat162float(so[row0 + mt * 16 + g + 8]);
         }
+        if (NT % 2 == 0 && d.wide) {         // upper window in n-tiles [0, NT / 2), lower window of the same tokens behind
+            constexpr int H = NT / 2;
+            const float lo_scale = pow2i(-kLoShift);
+#pragma unroll
+            for (int nt = 0; nt < H; ++nt)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int n = nt * 8 + tq * 2 + i;
+                    if (n < ntok) {
+                        const float hs = A.hscale[pos0 + n];
+                        yp[(size_t)(pos0 + n) * C + row0 + mt * 16 + g] = fmaf(sum[nt + H][i], lo_scale, sum[nt][i]) * hs * so0;
+                        yp[(size_t)(pos0 + n) * C + row0 + mt * 16 + g + 8] = fmaf(sum[nt + H][2 + i], lo_scale, sum[nt][2 + i]) * hs * so1;
+                    }
+                }
+            return;
+        }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -444,7 +473,11 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
                 const float xs = A.xscale[tok];
                 const float u = sum[nt][i] * (xs * s_u), gt = sum[nt][2 + i] * (xs * s_g);
                 const float h = A.act_on_w1 ? silu(u) * gt : silu(gt) * u;
-                A.h16[(size_t)pos * R + r] = __float2half_rn(fminf(fmaxf(h * s_h * pow2i(f), -65504.f), 65504.f));
+                const float v = h * s_h * pow2i(f);
+                const __half hi = __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f));
+                A.h16[(size_t)pos * R + r] = hi;
+                if (d.wide)
+                    A.h16lo[(size_t)pos * R + r] = __float2half_rn(fminf(fmaxf((v - __half2float(hi)) * pow2i(kLoShift), -65504.f), 65504.f));
             }
         }
     }
@@ -474,11 +507,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     const long u1 = unit_at(tab, cost * (blockIdx.x + 1) / gridDim.x, per_tb, w_full);
     const unsigned sA = (unsigned)__cvta_generic_to_shared(ringA);
 
-    // Describes the step that starts at unit v (valid = false past the end of this CTA's range).
-    auto decode = [&](long v) {
+    // Describes the step that starts at unit v (valid = false past the end of this CTA's range). S5 of a wide-range
+    // expert carries two fp16 windows per token, so a block of more than 16 tokens is taken as two steps over the
+    // same units: half 0 = its first 16 tokens, half 1 = the rest.
+    auto decode = [&](long v, int half) {
         StepDesc d;
         d.valid = v < u1;
-        d.nstep = 0; d.nt = 0; d.active = false; d.blob = nullptr; d.hexp = 0;
+        d.nstep = 0; d.nt = 0; d.active = false; d.blob = nullptr; d.hexp = 0; d.wide = false; d.last_half = true;
         d.row0 = d.k0 = d.klen = d.split = d.pos0 = d.ntok = 0;
         if (!d.valid) return d;
         const int tbg = (int)(v / per_tb);
@@ -496,6 +531,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         d.pos0 = A.offset[e] + tb * kTokBlock;
         d.ntok = min(kTokBlock, cnt - tb * kTokBlock);
         d.nt = (d.ntok + 7) >> 3;
+        d.wide = A.hexp[kMaxExperts + e] != 0;
+        if (DOWN && d.wide) {
+            d.last_half = half == 1 || d.ntok <= kTokBlock / 2;
+            d.pos0 += half * (kTokBlock / 2);
+            d.ntok = min(kTokBlock / 2, d.ntok - half * (kTokBlock / 2));
+            d.nt = 2 * ((d.ntok + 7) >> 3);
+        }
         d.blob = static_cast<const unsigned char*>(A.slots[A.slot_map[e]]);
         if (!DOWN) d.hexp = A.hexp[e];
         d.k0 = DOWN ? d.split * A.down_slice : 0;
@@ -505,7 +547,8 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         return d;
     };
 
-    StepDesc cur = decode(u);
+    int half = 0;
+    StepDesc cur = decode(u, 0);
     if (!cur.valid) { if (DOWN) { pdl_wait(); pdl_launch(); } return; }
     CopyState cs = DOWN ? start_step_weights<DOWN>(A, cur, sA) : start_step<DOWN>(A, cur, sA);
     if (DOWN) {
@@ -514,8 +557,8 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         start_step_acts(cs, cur);
     }
     while (cur.valid) {
-        u += cur.nstep;
-        const StepDesc next = decode(u);
+        if (cur.last_half) { u += cur.nstep; half = 0; } else half = 1;
+        const StepDesc next = decode(u, half);
         CopyState cs_next = cs;
         switch (cur.nt) {
             case 1: ffn_step<DOWN, 1>(A, cur, cs, next, cs_next, ringA); break;
@@ -627,6 +670,7 @@ FfnArgs make_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) {
     A.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
     A.x16 = ws_ptr<__half>(ctx, ctx->lay.x16);
     A.h16 = ws_ptr<__half>(ctx, ctx->lay.h16);
+    A.h16lo = ws_ptr<__half>(ctx, ctx->lay.h16lo);
     A.ypart = ws_ptr<float>(ctx, ctx->lay.ypart);
     A.R = ctx->cfg.ffn; A.C = ctx->cfg.hidden; A.act_on_w1 = ctx->cfg.act_on_w1;
     A.down_splits = ctx->down_splits; A.down_slice = ctx->down_slice;

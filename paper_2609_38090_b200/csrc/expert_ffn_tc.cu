@@ -85,7 +85,8 @@ struct TcArgs {
     void* const* slots; const int32_t* slot_map; const Sched* sched;
     const int32_t* count; const int32_t* offset;
     const float* xs_pos; const float* hm_pos; const float* sum_pos; const float* hscale;
-    __half* h16; float* ypart;
+    const int32_t* hexp;        // [2][kMaxExperts]: exponent of the intermediate's magnitude, then the wide-range flag
+    __half* h16; __half* h16lo; float* ypart;
     int32_t* status;
     int R, C, act_on_w1;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
@@ -180,7 +181,10 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const unsigned (&v)[32
 // The up/gate kernel may feed the codes as fp16 subnormals (code + 128) * 2^-24 and undo offset and scale in its
 // epilogue with the per-token sum of the activations: two fewer instructions per four weights in the converters.
 // The subtracted term grows with the sum of a token's activations, so batches that hold a token whose sum is large
-// against its norm (the schedule's dc_heavy flag) take the exact conversion, as the down kernel always does.
+// against its norm (the schedule's dc_heavy flag) take the exact conversion, as the down kernel always does. So do
+// the tiles of wide-range experts: the offset is 128 per code whatever the code, so rows whose codes are small
+// (a row triple whose scale is set by one large weight or by another matrix's row) lose the bits the offset takes
+// (measured: 1e-2 on a layer whose gate codes are mostly 0 and +-1).
 
 __device__ __forceinline__ unsigned cvt_exact_lo(unsigned u) {      // bytes 0,1 of (code + 128) -> half2 of codes
     unsigned v = __byte_perm(u, 0x64646464u, 0x4140);
@@ -195,10 +199,10 @@ __device__ __forceinline__ unsigned cvt_exact_hi(unsigned u) {      // bytes 2,3
 __device__ __forceinline__ float pow2_f(int e) { return __uint_as_float((unsigned)(max(-126, min(127, e)) + 127) << 23); }
 __device__ __forceinline__ int expo_f(float v) { return (int)((__float_as_uint(v) >> 23) & 0xff) - 127; }
 
-struct Tile { int pos0, ntok, row0; const unsigned char* blob; };
+struct Tile { int pos0, ntok, row0, wide; const unsigned char* blob; };
 
 template <bool DOWN, typename TC>
-__global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs A, const __grid_constant__ TileMaps bmaps) {
+__global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs A, const __grid_constant__ TileMaps bmaps, const __grid_constant__ TileMaps bmaps_lo) {
     constexpr int kTileN = TC::kTileN, kAStages = TC::kStages, kBStages = TC::kStages, kBTileBytes = TC::kBTileBytes;
     constexpr int kGroups = TC::kGroups, kAccBufs = TC::kAccBufs;
     constexpr int kEpiWarp0 = TC::kEpiWarp0, kTmaWarp = TC::kTmaWarp, kMmaWarp = TC::kMmaWarp, kIssuers = TC::kIssuers;
@@ -210,6 +214,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     __shared__ volatile int s_abort;
     __shared__ int s_ntile[kMaxExperts + 1];          // exclusive prefix of token tiles per active expert
     __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts];
+    __shared__ int s_wide[kMaxExperts];               // wide-range expert: two fp16 windows of the intermediate (see kLoShift)
     __shared__ const unsigned char* s_blob[kMaxExperts];
     __shared__ int s_nact;
 
@@ -233,11 +238,12 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 
     // per-expert table: one round of parallel loads, then a serial prefix over shared memory
     const int n_active = A.sched->n_active;
-    const bool subnormal = !DOWN && (A.up_conversion == 2 || (A.up_conversion == 0 && A.sched->dc_heavy == 0));
+    const bool sub_batch = !DOWN && (A.up_conversion == 2 || (A.up_conversion == 0 && A.sched->dc_heavy == 0));
     if (tid < kMaxExperts && tid < n_active) {
         const int e = A.sched->act_expert[tid];
         s_cnt[tid] = A.count[e];
         s_off[tid] = A.offset[e];
+        s_wide[tid] = A.hexp[kMaxExperts + e];
         s_blob[tid] = static_cast<const unsigned char*>(A.slots[A.slot_map[e]]);
     }
     if (tid == 0) {
@@ -254,7 +260,11 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     __syncthreads();
     if (tid == 0) {
         int acc = 0;
-        for (int a = 0; a < n_active; ++a) { s_ntile[a] = acc; acc += (s_cnt[a] + kTileN - 1) / kTileN; }
+        // S5 of a wide-range expert holds both windows of a token in one tile: half as many tokens per tile
+        for (int a = 0; a < n_active; ++a) {
+            const int tn = (DOWN && s_wide[a]) ? kTileN / 2 : kTileN;
+            s_ntile[a] = acc; acc += (s_cnt[a] + tn - 1) / tn;
+        }
         s_ntile[n_active] = acc;
     }
     tc_fence_before();
@@ -277,8 +287,10 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
         const int nt_e = s_ntile[lo + 1] - s_ntile[lo];
         const long local = tile - (long)s_ntile[lo] * n_mb;
         const int nb = (int)(local % nt_e), mb = (int)(local / nt_e);
-        t.pos0 = s_off[lo] + nb * kTileN;
-        t.ntok = min(kTileN, s_cnt[lo] - nb * kTileN);
+        t.wide = s_wide[lo];
+        const int tn = (DOWN && t.wide) ? kTileN / 2 : kTileN;
+        t.pos0 = s_off[lo] + nb * tn;
+        t.ntok = min(tn, s_cnt[lo] - nb * tn);
         t.row0 = mb * (DOWN ? kTileM : kTileM / 2);
         t.blob = s_blob[lo];
         return t;
@@ -335,7 +347,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
                         const unsigned u = w4[jj] ^ 0x80808080u;
-                        if (subnormal) {                      // u * 2^-24 as an fp16 subnormal: no subtraction here
+                        if (sub_batch && !t.wide) {           // u * 2^-24 as an fp16 subnormal: no subtraction here
                             f[q * 8 + jj * 2] = __byte_perm(u, 0u, 0x4140);
                             f[q * 8 + jj * 2 + 1] = __byte_perm(u, 0u, 0x4342);
                         } else {
@@ -378,6 +390,14 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                     uint32_t v[32];
                     __syncwarp();
                     tmem_ld32(acc_t + c0, v);
+                    if (t.wide) {                     // the lower window's sums sit one box further, scaled by 2^kLoShift
+                        uint32_t w[32];
+                        __syncwarp();
+                        tmem_ld32(acc_t + ncol + c0, w);
+                        const float lo_scale = pow2_f(-kLoShift);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(__uint_as_float(w[j]), lo_scale, __uint_as_float(v[j])));
+                    }
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int n = c0 + j;
@@ -404,14 +424,21 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                         const int pc = t.pos0 + min(n, t.ntok - 1);
                         const float xs = __ldg(A.xs_pos + pc);
                         float ru = odd ? ob : a, rg = odd ? b : oa;
-                        if (subnormal) {                      // undo the 2^-24 and the +128 offset of the codes
+                        if (sub_batch && !t.wide) {           // undo the 2^-24 and the +128 offset of the codes
                             const float off = -128.f * __ldg(A.sum_pos + pc);
                             ru = fmaf(ru, 16777216.f, off); rg = fmaf(rg, 16777216.f, off);
                         }
                         const float u = ru * (xs * s_u), g = rg * (xs * s_g);
                         const float act = A.act_on_w1 ? u : g, lin = A.act_on_w1 ? g : u;
                         const float h = __fdividef(act, 1.f + __expf(-act)) * lin;
-                        if (n < t.ntok) A.h16[(size_t)(t.pos0 + n) * R + r] = __float2half_rn(fminf(fmaxf(h * s_h * __ldg(A.hm_pos + pc), -65504.f), 65504.f));
+                        if (n < t.ntok) {
+                            const float val = h * s_h * __ldg(A.hm_pos + pc);
+                            const __half hi16 = __float2half_rn(fminf(fmaxf(val, -65504.f), 65504.f));
+                            A.h16[(size_t)(t.pos0 + n) * R + r] = hi16;
+                            if (t.wide)
+                                A.h16lo[(size_t)(t.pos0 + n) * R + r] =
+                                    __float2half_rn(fminf(fmaxf((val - __half2float(hi16)) * pow2_f(kLoShift), -65504.f), 65504.f));
+                        }
                     }
                 }
             }
@@ -429,7 +456,9 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 const Tile t = decode(tile);
                 const int hi = (t.ntok + kBoxStep - 1) / kBoxStep - 1;              // box of 32 (hi + 1) positions
                 const uint64_t map = reinterpret_cast<uint64_t>(&bmaps.m[hi]);
+                const uint64_t map_lo = reinterpret_cast<uint64_t>(&bmaps_lo.m[hi]);
                 const uint32_t box_bytes = (uint32_t)(hi + 1) * kBoxStep * kKB * 2;
+                const bool two = DOWN && t.wide;                                    // second box: the lower window, behind the first
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(b_empty(st), ph, &s_abort, A.spin_limit)) { ok = false; break; }
@@ -438,9 +467,12 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                         continue;
                     }
                     const uint32_t dst = b_s + st * kBTileBytes, bar = b_full(st);
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(box_bytes) : "memory");
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(two ? 2 * box_bytes : box_bytes) : "memory");
                     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
                                  ::"r"(dst), "l"(map), "r"(kb * kKB), "r"(t.pos0), "r"(bar) : "memory");
+                    if (two)
+                        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                                     ::"r"(dst + box_bytes), "l"(map_lo), "r"(kb * kKB), "r"(t.pos0), "r"(bar) : "memory");
                     if (++st == kBStages) { st = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -459,7 +491,8 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
             bool ready = false;                          // this issuer's next stage was already seen full
             for (long tile = blockIdx.x; tile < total && !s_abort; tile += gridDim.x) {
                 const Tile t = decode(tile);
-                const uint32_t idesc = make_idesc((t.ntok + 15) & ~15);
+                // columns of the MMA: the tile's tokens, or for a wide-range expert's down projection both boxes
+                const uint32_t idesc = make_idesc((DOWN && t.wide) ? 2 * ((t.ntok + kBoxStep - 1) / kBoxStep) * kBoxStep : (t.ntok + 15) & ~15);
                 if (!mbar_wait(acc_empty(buf), pacc, &s_abort, A.spin_limit)) break;   // its previous epilogue is done
                 tc_fence_after();
                 const uint32_t d_t = tmem + buf * kTileN;
@@ -561,6 +594,8 @@ TcArgs make_tc_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) 
     A.sum_pos = ws_ptr<float>(ctx, ctx->lay.sum_pos);
     A.hscale = ws_ptr<float>(ctx, ctx->lay.hscale);
     A.h16 = ws_ptr<__half>(ctx, ctx->lay.h16);
+    A.h16lo = ws_ptr<__half>(ctx, ctx->lay.h16lo);
+    A.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
     A.ypart = ws_ptr<float>(ctx, ctx->lay.ypart);
     A.status = ws_ptr<int32_t>(ctx, ctx->lay.status);
     A.R = ctx->cfg.ffn; A.C = ctx->cfg.hidden; A.act_on_w1 = ctx->cfg.act_on_w1;
@@ -587,9 +622,11 @@ bool build_tensor_maps(mira_ctx* ctx) {
     const EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fn);
     __half* x16p = ws_ptr<__half>(ctx, ctx->lay.x16p);
     __half* h16 = ws_ptr<__half>(ctx, ctx->lay.h16);
+    __half* h16lo = ws_ptr<__half>(ctx, ctx->lay.h16lo);
     for (int i = 0; i < kBoxMaps; ++i)
         if (!encode_map(enc, ctx->tmap_x16p[i], x16p, P, ctx->cfg.hidden, (i + 1) * kBoxStep) ||
-            !encode_map(enc, ctx->tmap_h16[i], h16, P, ctx->cfg.ffn, (i + 1) * kBoxStep))
+            !encode_map(enc, ctx->tmap_h16[i], h16, P, ctx->cfg.ffn, (i + 1) * kBoxStep) ||
+            !encode_map(enc, ctx->tmap_h16lo[i], h16lo, P, ctx->cfg.ffn, (i + 1) * kBoxStep))
             return false;
     return true;
 }
@@ -598,9 +635,11 @@ bool build_tensor_maps(mira_ctx* ctx) {
 template <bool DOWN, typename TC>
 static void launch_cfg(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps)[128], cudaStream_t st) {
     static_assert(TC::kTileN <= kBoxStep * kBoxMaps, "no box covers the tile");
-    TileMaps tm;
+    static_assert((TC::kTileN / 2) % kBoxStep == 0, "a wide-range expert's half tile is a whole number of boxes");
+    TileMaps tm, tm_lo;
     memcpy(&tm, maps, sizeof(tm));
-    launch_pdl(k_ffn_tc<DOWN, TC>, dim3(ctx->n_sm * TC::kCtasPerSm), dim3(TC::kThreads), TC::kSmem, st, A, tm);
+    memcpy(&tm_lo, ctx->tmap_h16lo, sizeof(tm_lo));          // only the down projection of wide-range experts reads it
+    launch_pdl(k_ffn_tc<DOWN, TC>, dim3(ctx->n_sm * TC::kCtasPerSm), dim3(TC::kThreads), TC::kSmem, st, A, tm, tm_lo);
 }
 
 // Estimated cost of a down projection in a 2-CTA layout with tiles of `tn` tokens: the kernel has few row tiles

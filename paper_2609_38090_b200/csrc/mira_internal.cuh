@@ -15,6 +15,11 @@ constexpr int kMaxTopK = 16;
 constexpr int kTokBlock = 32;      // tokens of one expert handled by one work item (4 MMA n-tiles)
 constexpr int kChunk = 64;         // reduction-dimension bytes of one weight row per pipeline stage
 constexpr int kDownSlice = 4096;   // nominal reduction length of one split of the down projection
+// The fp16 intermediate v = s_r h_r 2^f of a wide-range expert is kept as two fp16 values, hi = fp16(v) and
+// lo = fp16((v - hi) * 2^kLoShift), both saturating: together they hold 11 bits or more of every |v| in
+// [2^-38, 2^16). The down projection multiplies both by the same weight fragments and adds the second sum scaled
+// by 2^-kLoShift.
+constexpr int kLoShift = 24;
 
 // Device-resident schedule written by the grouping kernel and read by the expert kernels.
 struct Sched {
@@ -71,7 +76,9 @@ struct Layout {
     size_t xnorm;       // float [Tmax]   Euclidean norm of token t
     size_t xsum;        // float [Tmax]   sum of the fp16 activations of token t
     size_t hscale;      // float [Pmax]   2^-f_p that undoes the per-pair scaling of the fp16 intermediate
-    size_t hexp;        // int32 [Et]     per expert: exponent of the intermediate's expected magnitude per unit of |x|^2
+    size_t hexp;        // int32 [2][kMaxExperts] per expert: exponent of the intermediate's expected magnitude per unit of
+                        //                |x|^2; then 1 if the expert keeps a second (lower) window of its fp16 intermediate
+    size_t h16lo;       // half  [Pmax][R] the lower window of the intermediate (wide-range experts only)
     size_t x16;         // half  [Tmax][C]
     size_t x16p;        // half  [Pmax][C] activations in position order (tensor-core path only)
     size_t xs_pos;      // float [Pmax]    per position: undo factor of the token's fp16 pre-scaling (tensor-core path)
@@ -99,6 +106,7 @@ struct ProfRec { int id; cudaEvent_t a, b; };
 struct mira_ctx {
     alignas(64) unsigned char tmap_x16p[6][128];   // CUtensorMaps of x16p (tensor-core path): boxes of 32, 64, ..., 192 rows
     alignas(64) unsigned char tmap_h16[6][128];    // CUtensorMaps of h16, likewise
+    alignas(64) unsigned char tmap_h16lo[6][128];  // CUtensorMaps of h16lo, likewise
     bool tensor_path_ok = false;
     bool force_decode_path = false;
     int tc_layout = 0;                 // 0: chosen per step; 1..3 force a tile layout of the tensor-core kernels (MIRA_OPT_TENSOR_LAYOUT)

@@ -366,8 +366,17 @@ __device__ __forceinline__ int dc_heavy_tokens(const SchedArgs& S) {
 // Statistics CTA of expert e (every thread of the CTA calls it): the largest row scale of the blob in the expert's
 // slot, as the exponent the SwiGLU epilogues use to place the fp16 intermediate. Shared scale: the intermediate
 // s_r h_r grows like s^3; per-matrix scales: like s1 * s3. Experts without a slot, or outside the wave, are skipped.
+__device__ __forceinline__ float max8_bf16(const uint4& v) {
+    return fmaxf(fmaxf(fmaxf(bf16lo(v.x), bf16hi(v.x)), fmaxf(bf16lo(v.y), bf16hi(v.y))),
+                 fmaxf(fmaxf(bf16lo(v.z), bf16hi(v.z)), fmaxf(bf16lo(v.w), bf16hi(v.w))));
+}
+__device__ __forceinline__ float min8_bf16(const uint4& v) {
+    return fminf(fminf(fminf(bf16lo(v.x), bf16hi(v.x)), fminf(bf16lo(v.y), bf16hi(v.y))),
+                 fminf(fminf(bf16lo(v.z), bf16hi(v.z)), fminf(bf16lo(v.w), bf16hi(v.w))));
+}
+
 __device__ __forceinline__ void expert_stats(const SchedArgs& S, int e) {
-    __shared__ float s_m[2][32];
+    __shared__ float s_m[4][32];
     const bool sel = (S.mask.w[e >> 5] >> (e & 31)) & 1u;
     const int slot = (S.slots != nullptr && S.slot_map != nullptr && sel) ? S.slot_map[e] : -1;
     if (slot < 0) return;
@@ -375,28 +384,34 @@ __device__ __forceinline__ void expert_stats(const SchedArgs& S, int e) {
     const BlobFmt f = blob_fmt(S.per_matrix ? MIRA_FORMAT_PER_MATRIX : MIRA_FORMAT_SHARED, S.R, S.C);
     const uint4* su = reinterpret_cast<const uint4*>(blob + f.s_up);
     const uint4* sg = reinterpret_cast<const uint4*>(blob + f.s_gate);
-    float m1 = 0.f, m3 = 0.f;
+    float m1 = 0.f, m3 = 0.f, n1 = INFINITY, n3 = INFINITY;      // largest and smallest row scale (scales are positive)
     for (int i = threadIdx.x; i < S.R / 8; i += blockDim.x) {
         const uint4 v = __ldg(su + i);
-        m1 = fmaxf(m1, fmaxf(fmaxf(fmaxf(bf16lo(v.x), bf16hi(v.x)), fmaxf(bf16lo(v.y), bf16hi(v.y))),
-                             fmaxf(fmaxf(bf16lo(v.z), bf16hi(v.z)), fmaxf(bf16lo(v.w), bf16hi(v.w)))));
+        m1 = fmaxf(m1, max8_bf16(v)); n1 = fminf(n1, min8_bf16(v));
         if (S.per_matrix) {
             const uint4 w = __ldg(sg + i);
-            m3 = fmaxf(m3, fmaxf(fmaxf(fmaxf(bf16lo(w.x), bf16hi(w.x)), fmaxf(bf16lo(w.y), bf16hi(w.y))),
-                                 fmaxf(fmaxf(bf16lo(w.z), bf16hi(w.z)), fmaxf(bf16lo(w.w), bf16hi(w.w)))));
+            m3 = fmaxf(m3, max8_bf16(w)); n3 = fminf(n3, min8_bf16(w));
         }
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) {
-        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
-        m3 = fmaxf(m3, __shfl_xor_sync(0xffffffffu, m3, o));
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o)); n1 = fminf(n1, __shfl_xor_sync(0xffffffffu, n1, o));
+        m3 = fmaxf(m3, __shfl_xor_sync(0xffffffffu, m3, o)); n3 = fminf(n3, __shfl_xor_sync(0xffffffffu, n3, o));
     }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    if (lane == 0) { s_m[0][warp] = m1; s_m[1][warp] = m3; }
+    if (lane == 0) { s_m[0][warp] = m1; s_m[1][warp] = m3; s_m[2][warp] = n1; s_m[3][warp] = n3; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < nwarps; ++w) { m1 = fmaxf(m1, s_m[0][w]); m3 = fmaxf(m3, s_m[1][w]); }
+        for (int w = 1; w < nwarps; ++w) {
+            m1 = fmaxf(m1, s_m[0][w]); m3 = fmaxf(m3, s_m[1][w]); n1 = fminf(n1, s_m[2][w]); n3 = fminf(n3, s_m[3][w]);
+        }
         S.hexp[e] = S.per_matrix ? expo_of(m1) + expo_of(m3) : 3 * expo_of(m1);
+        // Wide-range experts: the intermediate is placed by the LARGEST row scale, and one fp16 window holds rows
+        // whose terms are up to 2^12 smaller. With the row scales spread over more than 8x (terms grow like s^3;
+        // per-matrix scales: s1 * s3 over more than 64x) the rows that carry the down projection's sum may fall
+        // below that window, so such experts keep a second fp16 window 2^24 lower (see kLoShift in the expert
+        // kernels) and their down projection runs over both.
+        S.hexp[kMaxExperts + e] = S.per_matrix ? (m1 * m3 > 64.f * n1 * n3) : (m1 > 8.f * n1);
     }
 }
 

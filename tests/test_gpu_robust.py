@@ -83,3 +83,34 @@ def test_log_normal_row_scales(shape, T, force, fmt):
     res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k, fmt=fmt)
     out = _run(wl, sh, T, fmt=fmt, force=force).cpu().numpy()
     assert np.isfinite(out).all() and gate_a(out, res["out64"]) <= TOL
+
+
+def _outlier_rows(shape, e):
+    """The quantizer test's heavy recipe: up-projection rows scaled log-normally (sigma 2) with the gate rows left
+    alone, and one down-projection weight in a hundred nine times larger. In the shared format a row's scale then
+    follows its up row, the gate and down codes of the large rows shrink towards zero, and the rows that carry the
+    output are far smaller than the largest scale suggests."""
+    w1, w2, w3 = inputs.expert_weights(shape, e)
+    g = np.random.default_rng(100 + e)
+    w1 = w1 * np.exp(2 * g.standard_normal((shape.R, 1))).astype(np.float32)
+    w2[g.random(w2.shape) < 0.01] *= np.float32(9.0)
+    return w1, w2, w3
+
+
+def _outliers_in_two_experts(shape, e):
+    return _outlier_rows(shape, e) if e in (1, 2) else inputs.expert_weights(shape, e)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("T,force", [(8, False), (80, False), (80, True), (300, False)])
+@pytest.mark.parametrize("shape,gen", [("tiny", _outlier_rows), ("wide", _outlier_rows), ("tiny", _outliers_in_two_experts)])
+def test_outlier_rows_take_the_two_window_intermediate(shape, gen, T, force, fmt):
+    """Experts whose row scales spread over more than a factor of 8 keep their fp16 intermediate in two windows
+    (2^24 apart) and run the down projection over both; the others, in the same batch, stay on one."""
+    sh = inputs.TINY if shape == "tiny" else inputs.LayerShape("h2", C=1024, R=2048, E=4, k=2, T=T, seed=4)
+    wl = Workload(sh, T, gen=gen, fmt=fmt)
+    res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k, fmt=fmt)
+    out = _run(wl, sh, T, fmt=fmt, force=force).cpu().numpy()
+    assert np.isfinite(out).all() and gate_a(out, res["out64"]) <= TOL
+    out_bf16 = _run(wl, sh, T, fmt=fmt, force=force, fp32=False).float().cpu().numpy()
+    assert gate_b(out_bf16, res["out64"]) <= TOL and gate_c(out_bf16, res["out64"], bf16_output=True) <= TOL
