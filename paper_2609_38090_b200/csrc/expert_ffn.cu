@@ -62,6 +62,12 @@ __device__ __forceinline__ unsigned cvt_exact_hi(unsigned u) {
     return *reinterpret_cast<unsigned*>(&r);
 }
 
+// fp32 -> fp16, round to nearest even, values beyond the fp16 range go to +-65504 instead of infinity
+__device__ __forceinline__ unsigned short f32_to_f16_sat(float v) {
+    unsigned short h;
+    asm("cvt.rn.satfinite.f16.f32 %0, %1;\n" : "=h"(h) : "f"(v));
+    return h;
+}
 __device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); }
 __device__ __forceinline__ float pow2i(int e) { return __uint_as_float((unsigned)(max(-126, min(127, e)) + 127) << 23); }
 __device__ __forceinline__ int expo(float v) { return (int)((__float_as_uint(v) >> 23) & 0xff) - 127; }
@@ -474,10 +480,11 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
                 const float u = sum[nt][i] * (xs * s_u), gt = sum[nt][2 + i] * (xs * s_g);
                 const float h = A.act_on_w1 ? silu(u) * gt : silu(gt) * u;
                 const float v = h * s_h * pow2i(f);
-                const __half hi = __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f));
-                A.h16[(size_t)pos * R + r] = hi;
+                const unsigned short hi = f32_to_f16_sat(v);
+                reinterpret_cast<unsigned short*>(A.h16)[(size_t)pos * R + r] = hi;
                 if (d.wide)
-                    A.h16lo[(size_t)pos * R + r] = __float2half_rn(fminf(fmaxf((v - __half2float(hi)) * pow2i(kLoShift), -65504.f), 65504.f));
+                    reinterpret_cast<unsigned short*>(A.h16lo)[(size_t)pos * R + r] =
+                        f32_to_f16_sat((v - __half2float(__ushort_as_half(hi))) * pow2i(kLoShift));
             }
         }
     }

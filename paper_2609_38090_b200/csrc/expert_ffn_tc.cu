@@ -31,6 +31,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <type_traits>
 #include <cuda.h>
 #include "mira_internal.cuh"
 
@@ -196,10 +197,38 @@ __device__ __forceinline__ unsigned cvt_exact_hi(unsigned u) {      // bytes 2,3
     __half2 r = __hsub2(*reinterpret_cast<__half2*>(&v), __half2half2(__ushort_as_half(0x6480)));
     return *reinterpret_cast<unsigned*>(&r);
 }
+// fp32 -> fp16, round to nearest even, values beyond the fp16 range go to +-65504 instead of infinity
+__device__ __forceinline__ unsigned short f32_to_f16_sat(float v) {
+    unsigned short h;
+    asm("cvt.rn.satfinite.f16.f32 %0, %1;\n" : "=h"(h) : "f"(v));
+    return h;
+}
 __device__ __forceinline__ float pow2_f(int e) { return __uint_as_float((unsigned)(max(-126, min(127, e)) + 127) << 23); }
 __device__ __forceinline__ int expo_f(float v) { return (int)((__float_as_uint(v) >> 23) & 0xff) - 127; }
 
 struct Tile { int pos0, ntok, row0, wide; const unsigned char* blob; };
+
+// One MMA row's 64 codes of a K-block (shared memory, 64 bytes) -> 32 half2 in k order. SUB: as the fp16
+// subnormals (code + 128) * 2^-24, no subtraction here; else the signed codes, exactly.
+template <bool SUB>
+__device__ __forceinline__ void convert_row(unsigned (&f)[32], uint32_t saddr) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        unsigned w4[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3]) : "r"(saddr + q * 16));
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const unsigned u = w4[jj] ^ 0x80808080u;
+            if (SUB) {
+                f[q * 8 + jj * 2] = __byte_perm(u, 0u, 0x4140);
+                f[q * 8 + jj * 2 + 1] = __byte_perm(u, 0u, 0x4342);
+            } else {
+                f[q * 8 + jj * 2] = cvt_exact_lo(u);
+                f[q * 8 + jj * 2 + 1] = cvt_exact_hi(u);
+            }
+        }
+    }
+}
 
 template <bool DOWN, typename TC>
 __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs A, const __grid_constant__ TileMaps bmaps, const __grid_constant__ TileMaps bmaps_lo) {
@@ -307,6 +336,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
         uint32_t gbase = 0;                                                   // K-blocks of this CTA's earlier tiles
         for (long tile = blockIdx.x; tile < total && !s_abort; tile += gridDim.x, gbase += (uint32_t)nkb) {
             const Tile t = decode(tile);
+            const bool sub = sub_batch && !t.wide;              // offset subnormals or exact codes: per tile, see above
             // source of the row this lane copies in instruction 0 (MMA row 32 gw + (lane & 7)); instruction i is 8 MMA
             // rows further: + 8 rows of W2^ (S5) or + 4 expert-hidden rows of W1^ / W3^ (S4)
             const unsigned char* src;
@@ -339,23 +369,8 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 __syncwarp();                                     // the other lanes' copies of this stage have landed too
                 const int ws = j % kWStages;
                 unsigned f[32];                                   // 64 codes as fp16, in k order
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    unsigned w4[4];
-                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3])
-                                 : "r"(w_rd + ws * kWStage + q * 16));
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const unsigned u = w4[jj] ^ 0x80808080u;
-                        if (sub_batch && !t.wide) {           // u * 2^-24 as an fp16 subnormal: no subtraction here
-                            f[q * 8 + jj * 2] = __byte_perm(u, 0u, 0x4140);
-                            f[q * 8 + jj * 2 + 1] = __byte_perm(u, 0u, 0x4342);
-                        } else {
-                            f[q * 8 + jj * 2] = cvt_exact_lo(u);
-                            f[q * 8 + jj * 2 + 1] = cvt_exact_hi(u);
-                        }
-                    }
-                }
+                if (sub) convert_row<true>(f, w_rd + ws * kWStage);
+                else convert_row<false>(f, w_rd + ws * kWStage);
                 const uint32_t g = gbase + (uint32_t)(kb0 + kGroups * j);
                 const uint32_t st = g % kAStages;
                 if (!mbar_wait(a_empty(st), ((g / kAStages) & 1u) ^ 1u, &s_abort, A.spin_limit)) { ok = false; break; }
@@ -386,24 +401,29 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 const int c = t.row0 + row;
                 // per-matrix format: the scale of output column c (row c of W2^)
                 const float so = A.per_matrix ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(t.blob + blob_fmt(1, R, C).s_out)[c]) : 1.f;
-                for (int c0 = 0; c0 < ncol; c0 += 32) {
-                    uint32_t v[32];
-                    __syncwarp();
-                    tmem_ld32(acc_t + c0, v);
-                    if (t.wide) {                     // the lower window's sums sit one box further, scaled by 2^kLoShift
-                        uint32_t w[32];
+                auto store = [&](auto wide_c) {       // compiled with and without the second window, chosen per tile
+                    constexpr bool kWide = decltype(wide_c)::value;
+                    for (int c0 = 0; c0 < ncol; c0 += 32) {
+                        uint32_t v[32];
                         __syncwarp();
-                        tmem_ld32(acc_t + ncol + c0, w);
-                        const float lo_scale = pow2_f(-kLoShift);
+                        tmem_ld32(acc_t + c0, v);
+                        if (kWide) {                  // the lower window's sums sit one box further, scaled by 2^kLoShift
+                            uint32_t w[32];
+                            __syncwarp();
+                            tmem_ld32(acc_t + ncol + c0, w);
+                            const float lo_scale = pow2_f(-kLoShift);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(__uint_as_float(w[j]), lo_scale, __uint_as_float(v[j])));
-                    }
+                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(__uint_as_float(w[j]), lo_scale, __uint_as_float(v[j])));
+                        }
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int n = c0 + j;
-                        if (n < t.ntok) A.ypart[(size_t)(t.pos0 + n) * C + c] = __uint_as_float(v[j]) * (__ldg(A.hscale + t.pos0 + n) * so);
+                        for (int j = 0; j < 32; ++j) {
+                            const int n = c0 + j;
+                            if (n < t.ntok) A.ypart[(size_t)(t.pos0 + n) * C + c] = __uint_as_float(v[j]) * (__ldg(A.hscale + t.pos0 + n) * so);
+                        }
                     }
-                }
+                };
+                if (t.wide) store(std::integral_constant<bool, true>{});
+                else store(std::integral_constant<bool, false>{});
             } else {
                 // Even lanes hold U (W1^ row), odd lanes G (W3^ row) of the same expert-hidden row. Of every pair of
                 // columns the even lane finishes the even one and the odd lane the odd one, branch-free.
@@ -412,35 +432,45 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 const float s_g = A.per_matrix ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(t.blob + blob_fmt(1, R, C).s_gate)[r]) : s_u;
                 const float s_h = A.per_matrix ? 1.f : s_u;          // folded into the intermediate (shared format only)
                 const int odd = row & 1;
-                for (int c0 = 0; c0 < ncol; c0 += 32) {
-                    uint32_t v[32];
-                    __syncwarp();
-                    tmem_ld32(acc_t + c0, v);
+                // The loop is compiled in three forms (offset subnormals / exact codes; one or two fp16 windows) and
+                // the form is chosen per tile, so that no per-element branch sits in it.
+                auto finish = [&](auto sub_c, auto wide_c) {
+                    constexpr bool kSub = decltype(sub_c)::value, kWide = decltype(wide_c)::value;
+                    for (int c0 = 0; c0 < ncol; c0 += 32) {
+                        uint32_t v[32];
+                        __syncwarp();
+                        tmem_ld32(acc_t + c0, v);
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        const float a = __uint_as_float(v[2 * jj]), b = __uint_as_float(v[2 * jj + 1]);
-                        const float oa = __shfl_xor_sync(0xffffffffu, a, 1), ob = __shfl_xor_sync(0xffffffffu, b, 1);
-                        const int n = c0 + 2 * jj + odd;
-                        const int pc = t.pos0 + min(n, t.ntok - 1);
-                        const float xs = __ldg(A.xs_pos + pc);
-                        float ru = odd ? ob : a, rg = odd ? b : oa;
-                        if (sub_batch && !t.wide) {           // undo the 2^-24 and the +128 offset of the codes
-                            const float off = -128.f * __ldg(A.sum_pos + pc);
-                            ru = fmaf(ru, 16777216.f, off); rg = fmaf(rg, 16777216.f, off);
-                        }
-                        const float u = ru * (xs * s_u), g = rg * (xs * s_g);
-                        const float act = A.act_on_w1 ? u : g, lin = A.act_on_w1 ? g : u;
-                        const float h = __fdividef(act, 1.f + __expf(-act)) * lin;
-                        if (n < t.ntok) {
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const float a = __uint_as_float(v[2 * jj]), b = __uint_as_float(v[2 * jj + 1]);
+                            const float oa = __shfl_xor_sync(0xffffffffu, a, 1), ob = __shfl_xor_sync(0xffffffffu, b, 1);
+                            const int n = c0 + 2 * jj + odd;
+                            const int pc = t.pos0 + min(n, t.ntok - 1);
+                            const float xs = __ldg(A.xs_pos + pc);
+                            float ru = odd ? ob : a, rg = odd ? b : oa;
+                            if (kSub) {                       // undo the 2^-24 and the +128 offset of the codes
+                                const float off = -128.f * __ldg(A.sum_pos + pc);
+                                ru = fmaf(ru, 16777216.f, off); rg = fmaf(rg, 16777216.f, off);
+                            }
+                            const float u = ru * (xs * s_u), g = rg * (xs * s_g);
+                            const float act = A.act_on_w1 ? u : g, lin = A.act_on_w1 ? g : u;
+                            const float h = __fdividef(act, 1.f + __expf(-act)) * lin;
                             const float val = h * s_h * __ldg(A.hm_pos + pc);
-                            const __half hi16 = __float2half_rn(fminf(fmaxf(val, -65504.f), 65504.f));
-                            A.h16[(size_t)(t.pos0 + n) * R + r] = hi16;
-                            if (t.wide)
-                                A.h16lo[(size_t)(t.pos0 + n) * R + r] =
-                                    __float2half_rn(fminf(fmaxf((val - __half2float(hi16)) * pow2_f(kLoShift), -65504.f), 65504.f));
+                            const unsigned short hi16 = f32_to_f16_sat(val);
+                            if (n < t.ntok) {
+                                reinterpret_cast<unsigned short*>(A.h16)[(size_t)(t.pos0 + n) * R + r] = hi16;
+                                if (kWide)
+                                    reinterpret_cast<unsigned short*>(A.h16lo)[(size_t)(t.pos0 + n) * R + r] =
+                                        f32_to_f16_sat((val - __half2float(__ushort_as_half(hi16))) * pow2_f(kLoShift));
+                            }
                         }
                     }
-                }
+                };
+                using T1 = std::integral_constant<bool, true>;
+                using T0 = std::integral_constant<bool, false>;
+                if (t.wide) finish(T0{}, T1{});               // wide-range experts always take the exact codes
+                else if (sub_batch) finish(T1{}, T0{});
+                else finish(T0{}, T0{});
             }
             tc_fence_before();
             __syncwarp();
