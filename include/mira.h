@@ -256,8 +256,10 @@ mira_status mira_predict_mixture(mira_ctx* ctx, int32_t layer, const void* hidde
 /* Options. MIRA_OPT_FORCE_DECODE_PATH (value 0/1): run S4/S5 of every batch through the weight-streaming
  * mma.sync kernels, also for the batch sizes that would take the tcgen05 kernels (used by the
  * tests to compare the two paths). MIRA_OPT_TENSOR_LAYOUT (value 0..3): 0 lets every step choose the tile layout of
- * the tcgen05 kernels from its token count (the default); 1, 2, 3 force the narrow, wide or big layout, for tests
- * and tuning. MIRA_OPT_UP_CONVERSION (value 0..2): how the tcgen05 up/gate kernel turns int8 codes into fp16 operands
+ * the tcgen05 kernels from its token count (the default); 1, 2, 3 force the narrow, wide or big layout, 4 and 5 the
+ * two-SM kernel (tcgen05 cta_group::2: tiles of 256 MMA rows over a cluster of two CTAs, 192 tokens x 4 ring stages
+ * or 128 tokens x 8; needs ffn % 128 == 0 and hidden % 256 == 0, else the one-CTA layouts run), for tests and
+ * tuning. MIRA_OPT_UP_CONVERSION (value 0..2): how the tcgen05 up/gate kernel turns int8 codes into fp16 operands
  * (the weight-streaming kernels always convert exactly). 0 (the default) decides per batch on the device: codes go in
  * as (code + 128) * 2^-24 with the offset taken out afterwards, unless some token's activations have a sum so large
  * against their norm (hidden size * |sum x| > 24576 * |x|_2) that the subtraction would cost accuracy, in which case

@@ -336,7 +336,8 @@ class Mira:
         _check(mira_set_option(self._ctx, MIRA_OPT_FORCE_DECODE_PATH, int(on)), "mira_set_option")
 
     def tensor_layout(self, layout: int) -> None:
-        """0: chosen per step (default); 1, 2, 3: force the narrow, wide or big tile layout of the tensor-core kernels."""
+        """0: chosen per step (default); 1, 2, 3: force the narrow, wide or big tile layout of the tensor-core kernels;
+        4, 5: the two-SM (cta_group::2) kernel with 192-token tiles x 4 stages or 128-token tiles x 8 stages."""
         _check(mira_set_option(self._ctx, MIRA_OPT_TENSOR_LAYOUT, int(layout)), "mira_set_option")
 
     def up_conversion(self, mode: int) -> None:

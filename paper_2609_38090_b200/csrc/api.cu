@@ -363,7 +363,7 @@ mira_status mira_poll_status(mira_ctx* ctx, uint32_t* miss_mask_out, void* strea
 mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value) {
     if (!ctx) return MIRA_ERR_INVALID_ARG;
     if (option == MIRA_OPT_FORCE_DECODE_PATH) { ctx->force_decode_path = value != 0; return MIRA_OK; }
-    if (option == MIRA_OPT_TENSOR_LAYOUT && value >= 0 && value <= 3) { ctx->tc_layout = value; return MIRA_OK; }
+    if (option == MIRA_OPT_TENSOR_LAYOUT && value >= 0 && value <= 5) { ctx->tc_layout = value; return MIRA_OK; }
     if (option == MIRA_OPT_UP_CONVERSION && value >= 0 && value <= 2) { ctx->up_conversion = value; return MIRA_OK; }
     if (option == MIRA_OPT_TEST_WAIT_TIMEOUT) { ctx->test_wait_timeout = value != 0; return MIRA_OK; }
     return MIRA_ERR_INVALID_ARG;

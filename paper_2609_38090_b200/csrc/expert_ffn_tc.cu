@@ -566,6 +566,395 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// The same grouped GEMM with the MMA spread over a PAIR of SMs (tcgen05 cta_group::2): a cluster of two CTAs works
+// on tiles of 256 MMA rows x up to 192 tokens. Each CTA converts ITS 128 weight rows into its own tensor memory and
+// loads ITS half of the activation tile (the tile's first / second half of the positions, one plain TMA tensor load
+// per K-block and CTA, no multicast) into its own shared memory; one thread of the even CTA (the leader) issues
+// the MMAs for both SMs. Per SM and K-block the activation tile costs half the shared-memory traffic of the one-CTA
+// kernels (they are bound by it with two CTAs per SM), and one issuing thread's waits and commits serve two SMs.
+// Measured on B200 (Mixtral shape, 2048 tokens, us per kernel, pair / one-CTA layouts): up/gate 1111 / 1143, down
+// 630 / 541; 512 tokens 435 / 373 and 300 / 198. The pair's K-block period (0.46 us for 256 x 192 x 64) is that of
+// the one-CTA kernel per SM, whatever the ring depth (4 or 8 stages) and the tile width (128 or 192 tokens), and as
+// a one-CTA-per-SM cluster kernel it cannot overlap its neighbours in the stream. It is therefore not chosen by
+// default (MIRA_OPT_TENSOR_LAYOUT 4 and 5 select it); what it needed to run at all: remote arrivals as plain
+// mbarrier.arrive (a .release.cluster arrival per K-block cost 40 % of the kernel), one tcgen05.commit per CTA's
+// barrier, the peer's TMA load completing its bytes on the leader's barrier.
+//   barriers   full[s]      leader only: its 4 converter warps + the peer's 4 (remote arrivals) + the leader's
+//                           expect_tx; both CTAs' loads complete their bytes on it
+//              empty[s]     one in each CTA, each signalled by a tcgen05.commit of the leader: the stage of the A
+//                           ring (TMEM) and of the B ring (shared memory) of that CTA is free
+//              acc_full[b]  one in each CTA, likewise: the accumulator half in that CTA's TMEM is complete
+//              acc_empty[b] leader only: 4 local + 4 remote epilogue warps have drained their halves
+// Every wait is bounded as in the one-CTA kernels; both CTAs meet at a cluster barrier before tensor memory is
+// freed, because the leader's MMAs write the peer's tensor memory and read its shared memory.
+constexpr int kPairGroups = 2, kPairAcc = 2;
+constexpr int kPairEpiWarp0 = 4 * kPairGroups, kPairTmaWarp = kPairEpiWarp0 + 4, kPairMmaWarp = kPairEpiWarp0 + 5;
+constexpr int kPairIssuers = 2;                       // MMA-issuing warps of the leader, taking the K-blocks in turn
+constexpr int kPairThreads = (kPairMmaWarp + kPairIssuers) * 32;
+constexpr uint32_t kPairTmemCols = 512;
+constexpr int kHalfBoxStep = 16, kHalfBoxMaps = 6;                    // half-tile boxes of 16, 32, ..., 96 positions
+// TN tokens per tile, NS ring stages (A ring in TMEM, B ring in shared memory): two accumulators of TN columns and
+// NS stages of 32 columns fill the 512 TMEM columns either as (192, 4) or as (128, 8).
+template <int TN, int NS> struct PairCfg {
+    static constexpr int kTileN = TN, kStages = NS;
+    static constexpr uint32_t kTmemA = kPairAcc * TN;
+    static constexpr int kBHalfBytes = (TN / 2) * kKB * 2;           // one CTA's half of the activation tile, per stage
+    static constexpr size_t kSmem = (size_t)NS * kBHalfBytes + (size_t)kPairGroups * kWStages * kWStage + 1024;
+    static_assert(kTmemA + NS * 32 <= kPairTmemCols, "TMEM columns");
+    static_assert(TN / 2 <= kHalfBoxStep * kHalfBoxMaps && TN % 64 == 0, "boxes cover a half tile");
+};
+using PairWide = PairCfg<192, 4>;
+using PairDeep = PairCfg<128, 8>;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {       // shared::cluster address of saddr in CTA `rank`
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];\n" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void umma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma2_commit(uint32_t cluster_bar) {                   // a barrier of either CTA of the pair
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ uint32_t make_idesc_m(int m, int n) {
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct HalfMaps { CUtensorMap m[kHalfBoxMaps]; };
+
+template <bool DOWN, typename PC>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+k_ffn_tc_pair(TcArgs A, const __grid_constant__ HalfMaps bmaps, const __grid_constant__ HalfMaps bmaps_lo) {
+    constexpr int kPairTileN = PC::kTileN, kPairStages = PC::kStages, kPairBHalfBytes = PC::kBHalfBytes;
+    constexpr uint32_t kPairTmemA = PC::kTmemA;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ uint64_t s_bar[2 * kPairStages + 6];   // full, empty, acc_full[2], acc_empty[2], turn[2]
+    __shared__ uint32_t s_tmem;
+    __shared__ volatile int s_abort;
+    __shared__ int s_ntile[kMaxExperts + 1];
+    __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts], s_wide[kMaxExperts];
+    __shared__ const unsigned char* s_blob[kMaxExperts];
+    __shared__ int s_nact;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_rank();             // 0: leader (issues the MMAs), 1: peer
+    const bool leader = rank == 0;
+    const int C = A.C, R = A.R;
+    const int K = DOWN ? R : C;
+    const int nkb = K / kKB;
+    const int n_mb = DOWN ? C / (2 * kTileM) : R / kTileM;       // row blocks of 256 MMA rows
+    const size_t per = (size_t)R * C;
+    const uint32_t b_s = smem_u32(smem);
+    const uint32_t w_s = b_s + kPairStages * kPairBHalfBytes;
+    const uint32_t bar0 = smem_u32(s_bar);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (kPairStages + s); };
+    auto acc_full = [&](int b) { return bar0 + 8u * (2 * kPairStages + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kPairStages + 2 + b); };
+    auto turn = [&](int q) { return bar0 + 8u * (2 * kPairStages + 4 + q); };
+
+    const int n_active = A.sched->n_active;
+    const bool sub_batch = !DOWN && (A.up_conversion == 2 || (A.up_conversion == 0 && A.sched->dc_heavy == 0));
+    if (tid < kMaxExperts && tid < n_active) {
+        const int e = A.sched->act_expert[tid];
+        s_cnt[tid] = A.count[e];
+        s_off[tid] = A.offset[e];
+        s_wide[tid] = A.hexp[kMaxExperts + e];
+        s_blob[tid] = static_cast<const unsigned char*>(A.slots[A.slot_map[e]]);
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(full(s), 4 + 4 + 1); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), kPairIssuers); mbar_init(acc_empty(b), 4 + 4); mbar_init(turn(b), 1); }
+        s_abort = 0;
+        s_nact = n_active;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == kPairTmaWarp) {                        // the same warp of both CTAs, as the pair allocation requires
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&s_tmem)), "r"(kPairTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;\n" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int a = 0; a < n_active; ++a) {
+            const int tn = (DOWN && s_wide[a]) ? kPairTileN / 2 : kPairTileN;
+            s_ntile[a] = acc; acc += (s_cnt[a] + tn - 1) / tn;
+        }
+        s_ntile[n_active] = acc;
+    }
+    tc_fence_before();
+    cluster_sync_all();                                // barriers of both CTAs are initialised before any remote arrival
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const long total = (long)s_ntile[s_nact] * n_mb;
+    const long pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    pdl_wait();
+    pdl_launch();
+
+    auto decode = [&](long tile) {
+        Tile t;
+        int lo = 0, hi = s_nact - 1;
+        while (lo < hi) { int mid = (lo + hi + 1) >> 1; if ((long)s_ntile[mid] * n_mb <= tile) lo = mid; else hi = mid - 1; }
+        const int nt_e = s_ntile[lo + 1] - s_ntile[lo];
+        const long local = tile - (long)s_ntile[lo] * n_mb;
+        const int nb = (int)(local % nt_e), mb = (int)(local / nt_e);
+        t.wide = s_wide[lo];
+        const int tn = (DOWN && t.wide) ? kPairTileN / 2 : kPairTileN;
+        t.pos0 = s_off[lo] + nb * tn;
+        t.ntok = min(tn, s_cnt[lo] - nb * tn);
+        t.row0 = mb * (DOWN ? 2 * kTileM : kTileM) + (int)rank * (DOWN ? kTileM : kTileM / 2);   // this CTA's first row
+        t.blob = s_blob[lo];
+        return t;
+    };
+    // Columns of the pair's MMA and what each CTA loads for them. Ordinary tile: N = the tokens rounded up to 32, the
+    // leader holds positions [0, N / 2), the peer [N / 2, N). Down projection of a wide-range expert: the leader holds
+    // the upper window of the tile's (at most 96) tokens, the peer the lower window of the same tokens, N / 2 each.
+    auto half_rows = [&](const Tile& t) {
+        return (DOWN && t.wide) ? ((t.ntok + 31) / 32) * 32 : ((t.ntok + 31) / 32) * 16;
+    };
+
+    if (warp < kPairEpiWarp0) {
+        // ------------------------------------------------ converters (as in the one-CTA kernel; the 'full' arrival goes to the leader)
+        const int group = warp >> 2, gw = warp & 3;
+        const uint32_t w_g = w_s + group * (kWStages * kWStage) + gw * kWWarp;
+        const uint32_t w_cp = w_g + (lane & 7) * kWRow + (lane >> 3) * 16;
+        const uint32_t w_rd = w_g + lane * kWRow;
+        uint32_t gbase = 0;
+        for (long tile = pair_id; tile < total && !s_abort; tile += n_pairs, gbase += (uint32_t)nkb) {
+            const Tile t = decode(tile);
+            const bool sub = sub_batch && !t.wide;
+            const unsigned char* src;
+            size_t src_step;
+            {
+                const int mrow = gw * 32 + (lane & 7);
+                if (DOWN) { src = t.blob + per + (size_t)(t.row0 + mrow) * R + (lane >> 3) * 16; src_step = (size_t)8 * R; }
+                else { src = t.blob + ((mrow & 1) ? 2 * per : 0) + (size_t)(t.row0 + (mrow >> 1)) * C + (lane >> 3) * 16; src_step = (size_t)4 * C; }
+            }
+            const int kb0 = (int)(((uint32_t)group + kPairGroups - gbase % kPairGroups) % kPairGroups);
+            const int nmine = (nkb - kb0 + kPairGroups - 1) / kPairGroups;
+#pragma unroll
+            for (int s = 0; s < kWStages - 1; ++s) {
+                if (s < nmine) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) cp_async16_s(w_cp + s * kWStage + i * 8 * kWRow, src + i * src_step + (size_t)(kb0 + kPairGroups * s) * kKB);
+                }
+                cp_async_commit();
+            }
+            bool ok = true;
+            for (int j = 0; j < nmine; ++j) {
+                const int pre = j + kWStages - 1;
+                if (pre < nmine) {
+                    const int ws = pre % kWStages;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) cp_async16_s(w_cp + ws * kWStage + i * 8 * kWRow, src + i * src_step + (size_t)(kb0 + kPairGroups * pre) * kKB);
+                }
+                cp_async_commit();
+                cp_async_wait<kWStages - 1>();
+                __syncwarp();
+                const int ws = j % kWStages;
+                unsigned f[32];
+                if (sub) convert_row<true>(f, w_rd + ws * kWStage);
+                else convert_row<false>(f, w_rd + ws * kWStage);
+                const uint32_t g = gbase + (uint32_t)(kb0 + kPairGroups * j);
+                const uint32_t st = g % kPairStages;
+                if (!mbar_wait(empty(st), ((g / kPairStages) & 1u) ^ 1u, &s_abort, A.spin_limit)) { ok = false; break; }
+                tc_fence_after();
+                __syncwarp();
+                tmem_st32(tmem + ((uint32_t)(gw * 32) << 16) + kPairTmemA + st * 32, f);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(full(st), 0));
+            }
+            cp_async_wait<0>();
+            if (!ok) break;
+        }
+    } else if (warp < kPairTmaWarp) {
+        // ------------------------------------------------ epilogue of this CTA's 128 accumulator rows
+        const int q4 = warp & 3, row = q4 * 32 + lane;
+        const uint32_t lane_base = tmem + ((uint32_t)(q4 * 32) << 16);
+        long it = 0;
+        for (long tile = pair_id; tile < total && !s_abort; tile += n_pairs, ++it) {
+            const Tile t = decode(tile);
+            const int buf = (int)(it % kPairAcc);
+            if (!mbar_wait(acc_full(buf), (uint32_t)((it / kPairAcc) & 1), &s_abort, A.spin_limit)) break;
+            tc_fence_after();
+            const uint32_t acc_t = lane_base + buf * kPairTileN;
+            const int hr = half_rows(t);
+            if (DOWN) {
+                const int c = t.row0 + row;
+                const float so = A.per_matrix ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(t.blob + blob_fmt(1, R, C).s_out)[c]) : 1.f;
+                const int ncol = t.wide ? hr : 2 * hr;            // columns that hold tokens (wide: the lower window follows)
+                auto store = [&](auto wide_c) {
+                    constexpr bool kWide = decltype(wide_c)::value;
+                    for (int c0 = 0; c0 < ncol; c0 += 32) {
+                        uint32_t v[32];
+                        __syncwarp();
+                        tmem_ld32(acc_t + c0, v);
+                        if (kWide) {
+                            uint32_t w[32];
+                            __syncwarp();
+                            tmem_ld32(acc_t + hr + c0, w);
+                            const float lo_scale = pow2_f(-kLoShift);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaf(__uint_as_float(w[j]), lo_scale, __uint_as_float(v[j])));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int n = c0 + j;
+                            if (n < t.ntok) A.ypart[(size_t)(t.pos0 + n) * C + c] = __uint_as_float(v[j]) * (__ldg(A.hscale + t.pos0 + n) * so);
+                        }
+                    }
+                };
+                if (t.wide) store(std::integral_constant<bool, true>{});
+                else store(std::integral_constant<bool, false>{});
+            } else {
+                const int r = t.row0 + (row >> 1);
+                const float s_u = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(t.blob + 3 * per)[r]);
+                const float s_g = A.per_matrix ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(t.blob + blob_fmt(1, R, C).s_gate)[r]) : s_u;
+                const float s_h = A.per_matrix ? 1.f : s_u;
+                const int odd = row & 1;
+                const int ncol = 2 * hr;
+                auto finish = [&](auto sub_c, auto wide_c) {
+                    constexpr bool kSub = decltype(sub_c)::value, kWide = decltype(wide_c)::value;
+                    for (int c0 = 0; c0 < ncol; c0 += 32) {
+                        uint32_t v[32];
+                        __syncwarp();
+                        tmem_ld32(acc_t + c0, v);
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const float a = __uint_as_float(v[2 * jj]), b = __uint_as_float(v[2 * jj + 1]);
+                            const float oa = __shfl_xor_sync(0xffffffffu, a, 1), ob = __shfl_xor_sync(0xffffffffu, b, 1);
+                            const int n = c0 + 2 * jj + odd;
+                            const int pc = t.pos0 + min(n, t.ntok - 1);
+                            const float xs = __ldg(A.xs_pos + pc);
+                            float ru = odd ? ob : a, rg = odd ? b : oa;
+                            if (kSub) {
+                                const float off = -128.f * __ldg(A.sum_pos + pc);
+                                ru = fmaf(ru, 16777216.f, off); rg = fmaf(rg, 16777216.f, off);
+                            }
+                            const float u = ru * (xs * s_u), g = rg * (xs * s_g);
+                            const float act = A.act_on_w1 ? u : g, lin = A.act_on_w1 ? g : u;
+                            const float h = __fdividef(act, 1.f + __expf(-act)) * lin;
+                            const float val = h * s_h * __ldg(A.hm_pos + pc);
+                            const unsigned short hi16 = f32_to_f16_sat(val);
+                            if (n < t.ntok) {
+                                reinterpret_cast<unsigned short*>(A.h16)[(size_t)(t.pos0 + n) * R + r] = hi16;
+                                if (kWide)
+                                    reinterpret_cast<unsigned short*>(A.h16lo)[(size_t)(t.pos0 + n) * R + r] =
+                                        f32_to_f16_sat((val - __half2float(__ushort_as_half(hi16))) * pow2_f(kLoShift));
+                            }
+                        }
+                    }
+                };
+                using T1 = std::integral_constant<bool, true>;
+                using T0 = std::integral_constant<bool, false>;
+                if (t.wide) finish(T0{}, T1{});
+                else if (sub_batch) finish(T1{}, T0{});
+                else finish(T0{}, T0{});
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0));
+        }
+    } else if (warp == kPairTmaWarp) {
+        // ------------------------------------------------ this CTA's half of the activation tile, one load per K-block
+        if (lane == 0) {
+            uint32_t st = 0, ph = 1;
+            const uint32_t full0 = map_to_cta(full(0), 0);        // the leader's 'full' barriers (8 bytes apart)
+            for (long tile = pair_id; tile < total && !s_abort; tile += n_pairs) {
+                const Tile t = decode(tile);
+                const int hr = half_rows(t);
+                const int mi = hr / kHalfBoxStep - 1;
+                const bool lo_window = DOWN && t.wide && !leader;
+                const uint64_t map = reinterpret_cast<uint64_t>(lo_window ? &bmaps_lo.m[mi] : &bmaps.m[mi]);
+                const int pos = (DOWN && t.wide) ? t.pos0 : t.pos0 + (int)rank * hr;
+                const uint32_t half_bytes = (uint32_t)hr * kKB * 2;
+                bool ok = true;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!mbar_wait(empty(st), ph, &s_abort, A.spin_limit)) { ok = false; break; }
+                    const uint32_t dst = b_s + st * kPairBHalfBytes, bar = full0 + 8u * st;
+                    if (leader)
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(full(st)), "r"(2 * half_bytes) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                                 ::"r"(dst), "l"(map), "r"(kb * kKB), "r"(pos), "r"(bar) : "memory");
+                    if (++st == kPairStages) { st = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (leader) {
+        // ------------------------------------------------ MMA issuers of the pair (one lane each, in the leader). Issuer q
+        // takes the K-blocks with running index g = q (mod 2); a turn barrier keeps the MMAs of a tile in K order, and
+        // one issuer's waits and commits run under the other's MMAs.
+        if (lane == 0) {
+            const int q = warp - kPairMmaWarp;
+            uint32_t g = 0, nmine = 0, buf = 0, pacc = 1;
+            const uint64_t bdesc0 = make_desc_sw128(b_s);
+            const uint32_t empty_peer0 = map_to_cta(empty(0), 1), acc_full_peer0 = map_to_cta(acc_full(0), 1);
+            bool ready = false;
+            for (long tile = pair_id; tile < total && !s_abort; tile += n_pairs) {
+                const Tile t = decode(tile);
+                const uint32_t idesc = make_idesc_m(2 * kTileM, 2 * half_rows(t));
+                if (!mbar_wait(acc_empty(buf), pacc, &s_abort, A.spin_limit)) break;
+                tc_fence_after();
+                const uint32_t d_t = tmem + buf * kPairTileN;
+                bool ok = true;
+                for (int kb = 0; kb < nkb; ++kb, ++g) {
+                    if (kPairIssuers == 2 && (int)(g & 1u) != q) continue;
+                    const uint32_t sa = g % kPairStages, pa = (g / kPairStages) & 1u;
+                    if (!ready && !mbar_wait(full(sa), pa, &s_abort, A.spin_limit)) { ok = false; break; }
+                    if (kPairIssuers == 2 && g > 0) {         // the other issuer has issued K-block g - 1
+                        const uint32_t n_other = (q == 0) ? nmine - 1 : nmine;
+                        if (!mbar_wait(turn(q), n_other & 1u, &s_abort, A.spin_limit)) { ok = false; break; }
+                    }
+                    tc_fence_after();
+                    const uint32_t a_t = tmem + kPairTmemA + sa * 32;
+                    const uint64_t bdesc = bdesc0 + (uint64_t)(sa * (kPairBHalfBytes >> 4));
+                    umma2_ts(d_t, a_t, bdesc, idesc, kb ? 1u : 0u);
+                    umma2_ts(d_t, a_t + 8, bdesc + 2, idesc, 1u);
+                    umma2_ts(d_t, a_t + 16, bdesc + 4, idesc, 1u);
+                    umma2_ts(d_t, a_t + 24, bdesc + 6, idesc, 1u);
+                    if (kPairIssuers == 2) mbar_arrive(turn(q ^ 1));
+                    umma2_commit(empty(sa));                       // both CTAs' stages are free once these MMAs have read them
+                    umma2_commit(empty_peer0 + 8u * sa);
+                    ++nmine;
+                    const uint32_t gn = g + kPairIssuers;
+                    ready = mbar_test(full(gn % kPairStages), (gn / kPairStages) & 1u);
+                }
+                if (!ok) break;
+                umma2_commit(acc_full(buf));
+                umma2_commit(acc_full_peer0 + 8u * buf);
+                if (++buf == kPairAcc) { buf = 0; pacc ^= 1u; }
+            }
+        }
+    }
+    // ---------------------------------------------------- common exit
+    tc_fence_before();
+    __syncthreads();
+    if (s_abort && tid == 0) atomicOr(A.status, 2);
+    cluster_sync_all();                                // the peer's tensor and shared memory are no longer in use by this CTA
+    if (warp == kPairTmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kPairTmemCols) : "memory");
+    }
+}
+
 // Position-ordered inputs of the tensor path, one block per position: x16p[pos] = x16[row_token[pos]] (so the
 // tokens of one expert are consecutive rows and one TMA box covers a token tile) and the per-position factors
 // of the SwiGLU epilogue: the undo factor of the token's fp16 pre-scaling and the power of two 2^f that places
@@ -658,6 +1047,11 @@ bool build_tensor_maps(mira_ctx* ctx) {
             !encode_map(enc, ctx->tmap_h16[i], h16, P, ctx->cfg.ffn, (i + 1) * kBoxStep) ||
             !encode_map(enc, ctx->tmap_h16lo[i], h16lo, P, ctx->cfg.ffn, (i + 1) * kBoxStep))
             return false;
+    for (int i = 0; i < kHalfBoxMaps; ++i)              // half-tile boxes of the two-SM kernels
+        if (!encode_map(enc, ctx->tmap_half[0][i], x16p, P, ctx->cfg.hidden, (i + 1) * kHalfBoxStep) ||
+            !encode_map(enc, ctx->tmap_half[1][i], h16, P, ctx->cfg.ffn, (i + 1) * kHalfBoxStep) ||
+            !encode_map(enc, ctx->tmap_half[2][i], h16lo, P, ctx->cfg.ffn, (i + 1) * kHalfBoxStep))
+            return false;
     return true;
 }
 
@@ -683,6 +1077,18 @@ static double down_cost(const mira_ctx* ctx, int tn, double tile_cost) {
     return std::ceil(tiles / (2.0 * ctx->n_sm)) * tile_cost;
 }
 
+// The two-SM kernel: one cluster of two CTAs per pair of SMs.
+template <bool DOWN>
+static void launch_pair(mira_ctx* ctx, const TcArgs& A, cudaStream_t st) {
+    static_assert(sizeof(HalfMaps) == sizeof(ctx->tmap_half[0]), "tensor map storage");
+    HalfMaps tm, tm_lo;
+    memcpy(&tm, ctx->tmap_half[DOWN ? 1 : 0], sizeof(tm));
+    memcpy(&tm_lo, ctx->tmap_half[2], sizeof(tm_lo));
+    if (ctx->tc_layout == 5) launch_pdl(k_ffn_tc_pair<DOWN, PairDeep>, dim3(ctx->n_sm / 2 * 2), dim3(kPairThreads), PairDeep::kSmem, st, A, tm, tm_lo);
+    else launch_pdl(k_ffn_tc_pair<DOWN, PairWide>, dim3(ctx->n_sm / 2 * 2), dim3(kPairThreads), PairWide::kSmem, st, A, tm, tm_lo);
+}
+static bool pair_shape_ok(const mira_config& c) { return c.ffn % kTileM == 0 && c.hidden % (2 * kTileM) == 0; }
+
 template <bool DOWN>
 static void launch_tc(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps)[128], cudaStream_t st) {
     // Up/gate has many row tiles (R / 64), so its time follows the number of tiles: narrow tiles while an expert gets
@@ -697,7 +1103,9 @@ static void launch_tc(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps
         if (DOWN) layout = 0.9 * down_cost(ctx, NarrowTile::kTileN, 1.0) <= down_cost(ctx, WideTile::kTileN, 1.3) ? 1 : 2;
         else layout = avg < kWideMinPerExpert ? 1 : (avg >= 256 && ctx->cfg.n_experts <= 16) ? 3 : 2;
     }
-    if (layout == 1) launch_cfg<DOWN, NarrowTile>(ctx, A, maps, st);
+    if (layout >= 4 && !pair_shape_ok(ctx->cfg)) layout = DOWN ? 2 : 3;
+    if (layout >= 4) launch_pair<DOWN>(ctx, A, st);
+    else if (layout == 1) launch_cfg<DOWN, NarrowTile>(ctx, A, maps, st);
     else if (layout == 3) launch_cfg<DOWN, BigTile>(ctx, A, maps, st);
     else launch_cfg<DOWN, WideTile>(ctx, A, maps, st);
 }
@@ -745,6 +1153,10 @@ mira_status set_tc_attributes() {
     MIRA_CUDA_OK(set_smem_attr<BigTile>());
     MIRA_CUDA_OK(set_smem_attr<WideTile>());
     MIRA_CUDA_OK(set_smem_attr<NarrowTile>());
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn_tc_pair<false, PairWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairWide::kSmem));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn_tc_pair<true, PairWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairWide::kSmem));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn_tc_pair<false, PairDeep>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairDeep::kSmem));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn_tc_pair<true, PairDeep>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairDeep::kSmem));
     return MIRA_OK;
 }
 

@@ -107,6 +107,7 @@ struct mira_ctx {
     alignas(64) unsigned char tmap_x16p[6][128];   // CUtensorMaps of x16p (tensor-core path): boxes of 32, 64, ..., 192 rows
     alignas(64) unsigned char tmap_h16[6][128];    // CUtensorMaps of h16, likewise
     alignas(64) unsigned char tmap_h16lo[6][128];  // CUtensorMaps of h16lo, likewise
+    alignas(64) unsigned char tmap_half[3][6][128]; // x16p, h16, h16lo with boxes of 16, 32, ..., 96 rows (two-SM kernels)
     bool tensor_path_ok = false;
     bool force_decode_path = false;
     int tc_layout = 0;                 // 0: chosen per step; 1..3 force a tile layout of the tensor-core kernels (MIRA_OPT_TENSOR_LAYOUT)

@@ -398,13 +398,15 @@ def test_many_experts_near_the_limits(T):
     _check_layer(wl, out.float().cpu().numpy(), res, False)
 
 
-@pytest.mark.parametrize("layout", [1, 2, 3])
-@pytest.mark.parametrize("shape", ["tiny", "small_shared"])
+@pytest.mark.parametrize("layout", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("shape", ["tiny", "small_shared", "pairs"])
 def test_every_tile_layout_of_the_tensor_core_kernels(layout, shape):
-    """Each tile layout forced in turn (narrow / wide / big) on batches with full, ragged and multi-tile experts;
-    left to itself a step only ever takes the layout its token count selects."""
-    sh = inputs.TINY if shape == "tiny" else SMALL_SHARED
-    for T in (70, 300):
+    """Each tile layout forced in turn (narrow / wide / big, and the two-SM kernel in both of its forms) on batches
+    with full, ragged and multi-tile experts; left to itself a step only ever takes the layout its token count
+    selects. ("small_shared" has sizes the two-SM kernel does not take: there layouts 4 and 5 must fall back.)"""
+    sh = {"tiny": inputs.TINY, "small_shared": SMALL_SHARED,
+          "pairs": inputs.LayerShape("pairs", C=512, R=384, E=5, k=2, T=300, n_shared=1, zipf_a=1.3, seed=17)}[shape]
+    for T in (70, 300, 900):
         wl, d, m, blobs, slots, slot_map = _setup(sh, T, out_fp32=True)
         m.tensor_layout(layout)
         out = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k)

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 TOL = 2e-3
 
 
-def _run(wl, sh, T, fmt=0, conversion=0, force=False, fp32=True):
+def _run(wl, sh, T, fmt=0, conversion=0, force=False, fp32=True, layout=0):
     from paper_2609_38090_b200 import binding as b
     d = wl.device_inputs()
     m = b.Mira(sh.C, sh.R, sh.E, n_shared=sh.n_shared, n_layers=4, max_tokens=T, max_top_k=sh.k, out_fp32=fp32, fmt=fmt)
@@ -23,6 +23,7 @@ def _run(wl, sh, T, fmt=0, conversion=0, force=False, fp32=True):
     assert np.array_equal(blobs.cpu().numpy(), np.stack(wl.blobs))
     m.up_conversion(conversion)
     m.force_decode_path(force)
+    m.tensor_layout(layout)
     slot_map = torch.arange(sh.E + sh.n_shared, dtype=torch.int32, device="cuda")
     out = m.moe_layer(d["x"], d["wr"], d["bias"], b.slot_table(blobs), slot_map, sh.k)
     torch.cuda.synchronize()
@@ -114,3 +115,16 @@ def test_outlier_rows_take_the_two_window_intermediate(shape, gen, T, force, fmt
     assert np.isfinite(out).all() and gate_a(out, res["out64"]) <= TOL
     out_bf16 = _run(wl, sh, T, fmt=fmt, force=force, fp32=False).float().cpu().numpy()
     assert gate_b(out_bf16, res["out64"]) <= TOL and gate_c(out_bf16, res["out64"], bf16_output=True) <= TOL
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("layout", [4, 5])
+def test_outlier_rows_on_the_two_sm_kernel(layout, fmt):
+    """The two windows of a wide-range expert on the cta_group::2 kernel: the leader CTA holds the upper window of a
+    tile's tokens, its peer the lower one."""
+    sh = inputs.TINY
+    for T in (80, 300):
+        wl = Workload(sh, T, gen=_outliers_in_two_experts, fmt=fmt)
+        res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k, fmt=fmt)
+        out = _run(wl, sh, T, fmt=fmt, layout=layout).cpu().numpy()
+        assert np.isfinite(out).all() and gate_a(out, res["out64"]) <= TOL
