@@ -260,11 +260,16 @@ def replica_throughput(tokens: int, steps: int, world: int, ms_total: float) -> 
     return world * tokens * steps / (ms_total / 1e3)
 
 
-def timed_blocks(fn, steps, barrier, dev, world, min_seconds=0.5, finish=None, max_blocks=400):
+MIN_SECONDS = 0.5      # every timed region lasts at least this long (--min-seconds; 0 = one block, for profiler runs)
+
+
+def timed_blocks(fn, steps, barrier, dev, world, min_seconds=None, finish=None, max_blocks=400):
     """Times blocks of exactly `steps` steps, each bracketed by barrier + synchronize on both sides and CUDA events
     on the launching stream, repeated until the blocks together last at least `min_seconds` (so that the clock
     sampler sees the timed region). Returns the per-block times in ms (max over ranks)."""
     import torch
+    if min_seconds is None:
+        min_seconds = MIN_SECONDS
     blocks, total = [], 0.0
     while True:
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -399,7 +404,7 @@ def measure_resident(layer: ResidentLayer, T: int, args, world, rank, sampler, b
 
     # per-kernel pass: the same steps with an event pair around every launch (the events switch the programmatic
     # launch overlap off, so the kernel times add up to a little more than the step)
-    n_prof = max(args.steps, min(400, int(0.1e3 / max(ms_step, 1e-3))))
+    n_prof = max(args.steps, min(400, int(0.1e3 / max(ms_step, 1e-3)))) if MIN_SECONDS > 0 else args.steps
     m.profile(True)
     barrier()
     for i in range(n_prof):
@@ -896,6 +901,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--ref-tokens", type=int, default=4, help="tokens of the bounded oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=0.5,
+                    help="repeat the block of --steps steps until the timed region lasts this long (0: one block)")
     ap.add_argument("--headline-only", action="store_true",
                     help="time the headline configuration only (the default run adds one record per other configuration)")
     ap.add_argument("--k-pred", type=int, default=4, help="stack workload: expert ids requested from each predictor head")
@@ -912,8 +919,9 @@ def main():
     ap.add_argument("--mode", default="resident", choices=["resident", "staged"],
                     help="staged: prefill with the predictor and a 4+2-slot expert cache fed from pinned host memory")
     args = ap.parse_args()
-    global FMT
+    global FMT, MIN_SECONDS
     FMT = 1 if args.format == "per-matrix" else 0
+    MIN_SECONDS = max(0.0, args.min_seconds)
     if FMT and (args.workload == "stack" or args.mode == "staged"):
         ap.error("--format per-matrix is available for the resident layer workloads")
     if args.warmup < 3 and args.impl == "mira":
