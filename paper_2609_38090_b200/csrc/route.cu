@@ -99,20 +99,6 @@ __device__ __forceinline__ float topk_softmax(float my_val, int k, int lane) {
     return p / z;
 }
 
-// Exclusive prefix sums over n <= 256 counts by ONE warp: lane l takes the contiguous chunk [l c, l c + c), c = ceil(n / 32).
-// Writes off[0..n] (off[n] = total). Called by all 32 lanes of a warp.
-__device__ __forceinline__ void warp_exclusive_offsets(const int* cnt, int* off, int n, int lane) {
-    const int c = (n + 31) >> 5, i0 = min(n, lane * c), i1 = min(n, i0 + c);
-    int sum = 0;
-    for (int i = i0; i < i1; ++i) sum += cnt[i];
-    int incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-    int run = incl - sum;
-    for (int i = i0; i < i1; ++i) { off[i] = run; run += cnt[i]; }
-    if (lane == 31) off[n] = incl;
-}
-
 // One CTA scores kScoreTok tokens against all E rows of W. Optionally: writes the fp16 copy of the
 // tokens pre-scaled by a power of two (so that any bf16 magnitude fits fp16 exactly) and selects
 // the top-k experts with their softmax weights.
@@ -304,7 +290,11 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
     }
     for (int s = threadIdx.x; s < ns; s += blockDim.x) s_count[E + s] = T;
     __syncthreads();
-    if (threadIdx.x < 32) warp_exclusive_offsets(s_count, s_off, E + ns, threadIdx.x);
+    if (threadIdx.x == 0) {
+        int a = 0;
+        for (int e = 0; e < E + ns; ++e) { s_off[e] = a; a += s_count[e]; }
+        s_off[E + ns] = a;
+    }
     __syncthreads();
     notify_host(G, s_count, E + ns);
     for (int e = threadIdx.x; e <= E + ns; e += blockDim.x) {
@@ -425,47 +415,26 @@ __device__ __forceinline__ void expert_stats(const SchedArgs& S, int e) {
     }
 }
 
-// Tail of the schedule, by one warp (all 32 lanes call it): the active experts in ascending order with the prefix sums
-// of their token blocks and of the blocks' costs. tb[i] = token blocks of expert i if it is active, else 0. Lane l
-// takes a contiguous chunk of the experts; four warp scans give every lane its first rank and its first prefix values.
-__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot, int dc_heavy, int lane) {
-    const int c = (Etot + 31) >> 5, i0 = min(Etot, lane * c), i1 = min(Etot, i0 + c);
+// Serial tail of the schedule (one thread): the active experts in ascending order with the prefix sums of their
+// token blocks and of the blocks' costs. tb[i] = token blocks of expert i if it is active, else 0.
+__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot, int dc_heavy) {
     int n = 0, a = 0, wu = 0, wd = 0;
-    for (int i = i0; i < i1; ++i) {
+    sched->dc_heavy = dc_heavy;
+    for (int i = 0; i < Etot; ++i) {
         const int b = tb[i];
         if (b > 0) {
+            sched->act_expert[n] = i; sched->tb_prefix[n] = a;
+            sched->w_prefix[0][n] = wu; sched->w_prefix[1][n] = wd;
             const int last = (count[i] - (b - 1) * kTokBlock + 7) >> 3;          // n-tiles of the last block, 1..4
             wu += (b - 1) * block_cost(0, 4) + block_cost(0, last);
             wd += (b - 1) * block_cost(1, 4) + block_cost(1, last);
             a += b; ++n;
         }
     }
-    int sn = n, sa = a, su = wu, sd = wd;                   // inclusive scans over the lanes
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int vn = __shfl_up_sync(0xffffffffu, sn, o), va = __shfl_up_sync(0xffffffffu, sa, o);
-        const int vu = __shfl_up_sync(0xffffffffu, su, o), vd = __shfl_up_sync(0xffffffffu, sd, o);
-        if (lane >= o) { sn += vn; sa += va; su += vu; sd += vd; }
-    }
-    n = sn - n; a = sa - a; wu = su - wu; wd = sd - wd;     // this lane's first rank and prefix values
-    for (int i = i0; i < i1; ++i) {
-        const int b = tb[i];
-        if (b > 0) {
-            sched->act_expert[n] = i; sched->tb_prefix[n] = a;
-            sched->w_prefix[0][n] = wu; sched->w_prefix[1][n] = wd;
-            const int last = (count[i] - (b - 1) * kTokBlock + 7) >> 3;
-            wu += (b - 1) * block_cost(0, 4) + block_cost(0, last);
-            wd += (b - 1) * block_cost(1, 4) + block_cost(1, last);
-            a += b; ++n;
-        }
-    }
-    if (lane == 31) {                                        // totals (sn, sa, su, sd are the sums over all lanes here)
-        sched->tb_prefix[sn] = sa;
-        sched->w_prefix[0][sn] = su; sched->w_prefix[1][sn] = sd;
-        sched->n_active = sn;
-        sched->total_tb = sa;
-        sched->dc_heavy = dc_heavy;
-    }
+    sched->tb_prefix[n] = a;
+    sched->w_prefix[0][n] = wu; sched->w_prefix[1][n] = wd;
+    sched->n_active = n;
+    sched->total_tb = a;
 }
 
 // Called by every thread of a CTA of at least kMaxExperts threads. Thread e looks at expert e; a warp covers one word
@@ -491,7 +460,7 @@ __device__ __forceinline__ void schedule_body(const SchedArgs& S, const int* cou
         }
     }
     const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
-    if (threadIdx.x < 32) write_schedule(S.sched, s_tb, count, Etot, heavy, threadIdx.x);    // s_tb is 0 for inactive experts
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, heavy);    // s_tb is 0 for inactive experts
 }
 
 // S3 for large batches, one CTA; with do_sched also the work schedule of a call that runs every routed expert.
@@ -594,27 +563,13 @@ __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, 
     if (lane == 0) { s_red[1][warp] = ss; s_red[2][warp] = sm; }
     // scores: warp w takes experts w, w + nwarps, ...
     const uint4* wg = reinterpret_cast<const uint4*>(A.W);
-    for (int e = warp; e < E; e += 2 * nwarps) {              // two rows of the router per pass, their loads in flight together
-        const int e2 = e + nwarps;
-        const bool two = e2 < E;
-        const uint4* r0 = wg + (size_t)e * c8;
-        const uint4* r1 = wg + (size_t)(two ? e2 : e) * c8;
-        float acc = 0.f, acc2 = 0.f;
-#pragma unroll 4
-        for (int i = lane; i < c8; i += 32) {
-            const uint4 w0 = __ldg(r0 + i), w1 = __ldg(r1 + i), xv = xs[i];
-            acc = dot8(w0, xv, acc);
-            acc2 = dot8(w1, xv, acc2);
-        }
+    for (int e = warp; e < E; e += nwarps) {
+        float acc = 0.f;
+#pragma unroll 8
+        for (int i = lane; i < c8; i += 32) acc = dot8(__ldg(wg + (size_t)e * c8 + i), xs[i], acc);
 #pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            acc2 += __shfl_xor_sync(0xffffffffu, acc2, o);
-        }
-        if (lane == 0) {
-            s_sc[e] = acc + (A.bias ? A.bias[e] : 0.f);
-            if (two) s_sc[e2] = acc2 + (A.bias ? A.bias[e2] : 0.f);
-        }
+        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) s_sc[e] = acc + (A.bias ? A.bias[e] : 0.f);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -803,7 +758,11 @@ __global__ void __launch_bounds__(kSingleCtaThreads) k_route_small(TokenArgs A, 
     }
     for (int s = threadIdx.x; s < ns; s += kSingleCtaThreads) s_count[E + s] = T;
     __syncthreads();
-    if (threadIdx.x < 32) warp_exclusive_offsets(s_count, s_off, Etot, threadIdx.x);
+    if (threadIdx.x == 0) {
+        int a = 0;
+        for (int e = 0; e < Etot; ++e) { s_off[e] = a; a += s_count[e]; }
+        s_off[Etot] = a;
+    }
     __syncthreads();
     notify_host(G, s_count, Etot);
     for (int e = threadIdx.x; e <= Etot; e += kSingleCtaThreads) {
@@ -833,7 +792,7 @@ __global__ void __launch_bounds__(kSingleCtaThreads) k_route_small(TokenArgs A, 
         }
     }
     const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
-    if (threadIdx.x < 32) write_schedule(S.sched, s_tb, s_count, Etot, heavy, threadIdx.x);
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot, heavy);
 }
 
 // S7 pooling: pooled[e] = mean_t score[t][e]; then the k_pred best pooled scores.
