@@ -266,8 +266,13 @@ mira_status mira_predict_mixture(mira_ctx* ctx, int32_t layer, const void* hidde
  * the codes are converted exactly; 1 forces the exact conversion, 2 the offset form (tests and tuning). MIRA_OPT_TEST_WAIT_TIMEOUT (value 1; test hook): the next tcgen05
  * up/gate launch of this context leaves out one activation load in its first CTA and gives up its waits after 4096
  * polls instead of 2^24, so that CTA takes the time-out path (status MIRA_ERR_TIMEOUT at the next poll); the option
- * clears itself with that launch. */
-enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2, MIRA_OPT_UP_CONVERSION = 3, MIRA_OPT_TEST_WAIT_TIMEOUT = 4 };
+ * clears itself with that launch. MIRA_OPT_HYBRID_MIN_UP / MIRA_OPT_HYBRID_MIN_DOWN (value >= -1): a step may split its
+ * experts between the two kernel families per projection: experts routed fewer than `value` pairs run on the
+ * weight-streaming kernel, the others on the tcgen05 kernel (0: all tensor-core, INT32_MAX: all streaming, -1: the
+ * library's rule for the step's token count, the default). Applies to steps of at least 16 tokens of a context whose
+ * shape the tensor-core kernels take; set it before the routing call of the step. */
+enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2, MIRA_OPT_UP_CONVERSION = 3, MIRA_OPT_TEST_WAIT_TIMEOUT = 4,
+       MIRA_OPT_HYBRID_MIN_UP = 5, MIRA_OPT_HYBRID_MIN_DOWN = 6 };
 mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value);
 
 /* ---------------------------------------------------------------------------------------------------------------

@@ -121,6 +121,8 @@ MIRA_OPT_FORCE_DECODE_PATH = 1
 MIRA_OPT_TENSOR_LAYOUT = 2
 MIRA_OPT_UP_CONVERSION = 3
 MIRA_OPT_TEST_WAIT_TIMEOUT = 4
+MIRA_OPT_HYBRID_MIN_UP = 5
+MIRA_OPT_HYBRID_MIN_DOWN = 6
 mira_profile_read = lib.mira_profile_read
 KERNEL_CLASSES = ("route", "group", "schedule", "up_gate", "down", "combine", "scores", "pool", "quantize", "unpack")
 mira_status_string = lib.mira_status_string
@@ -343,6 +345,12 @@ class Mira:
     def up_conversion(self, mode: int) -> None:
         """0: decided per batch on the device (default); 1: exact code conversion in the up/gate kernels; 2: offset subnormals."""
         _check(mira_set_option(self._ctx, MIRA_OPT_UP_CONVERSION, int(mode)), "mira_set_option")
+
+    def hybrid_min(self, up: int = -1, down: int = -1) -> None:
+        """Pair count from which an expert goes to the tcgen05 kernel of the up/gate and of the down projection
+        (-1: the library's rule; 0: all; 2**31 - 1: none). Set before the step's routing call."""
+        _check(mira_set_option(self._ctx, MIRA_OPT_HYBRID_MIN_UP, int(up)), "mira_set_option")
+        _check(mira_set_option(self._ctx, MIRA_OPT_HYBRID_MIN_DOWN, int(down)), "mira_set_option")
 
     def test_wait_timeout(self) -> None:
         """Test hook: the next tcgen05 up/gate launch takes its time-out path in one CTA (see MIRA_OPT_TEST_WAIT_TIMEOUT)."""

@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <new>
 #include <cstring>
+#include <climits>
 #include "mira_internal.cuh"
 
 namespace mira {
@@ -122,13 +123,16 @@ mira_status do_experts(mira_ctx* ctx, int T, void* const* slots, const int32_t* 
                        int final_wave, void* out, int schedule_done, cudaStream_t st) {
     mira_status s = MIRA_OK;
     if (!schedule_done && (s = launch_schedule(ctx, T, slots, slot_map, mask, mask == nullptr, st)) != MIRA_OK) return s;
-    // every wave of one routed batch takes the same kernels (T decides), so the partial-sum layout is consistent; the
-    // two projections switch to the tensor-core kernel at different sizes and share the fp16 intermediate's layout
-    const bool tc_ok = ctx->tensor_path_ok && !ctx->force_decode_path;
-    const bool tc_up = tc_ok && T >= tc_min_tokens_up(ctx->cfg), tc_down = tc_ok && T >= tc_min_tokens_down(ctx->cfg);
-    if ((s = tc_up ? launch_up_gate_tc(ctx, slots, slot_map, st) : launch_up_gate(ctx, slots, slot_map, st)) != MIRA_OK) return s;
-    if ((s = tc_down ? launch_down_tc(ctx, slots, slot_map, st) : launch_down(ctx, slots, slot_map, st)) != MIRA_OK) return s;
-    if (final_wave) s = launch_combine(ctx, T, ctx->route_k, tc_down ? 1 : ctx->down_splits, out, st);
+    // Every wave of one routed batch takes the same kernels (T and k decide), so the partial-sum layout is consistent.
+    // Per projection, the experts below the step's threshold run on the weight-streaming kernel and the others on the
+    // tensor-core kernel (the schedule was written for the same thresholds); both share the fp16 intermediate's layout.
+    int tc_min[2];
+    step_tc_min(ctx, T, ctx->route_k, tc_min);
+    if (tc_min[0] > 0 && (s = launch_up_gate(ctx, slots, slot_map, st)) != MIRA_OK) return s;
+    if (tc_min[0] < INT_MAX && (s = launch_up_gate_tc(ctx, slots, slot_map, st)) != MIRA_OK) return s;
+    if (tc_min[1] > 0 && (s = launch_down(ctx, slots, slot_map, st)) != MIRA_OK) return s;
+    if (tc_min[1] < INT_MAX && (s = launch_down_tc(ctx, slots, slot_map, st)) != MIRA_OK) return s;
+    if (final_wave) s = launch_combine(ctx, T, ctx->route_k, tc_min[1] > 0 ? ctx->down_splits : 1, tc_min[1], out, st);
     return s;
 }
 
@@ -153,8 +157,21 @@ mira_status run_scheduled_experts(mira_ctx* ctx, int T, void* const* slots, cons
 mira_status combine_only(mira_ctx* ctx, int T, void* out, cudaStream_t st) {
     if (!ctx || ctx->route_T != T || T < 1 || !out) return MIRA_ERR_INVALID_ARG;
     if (misaligned(out)) return MIRA_ERR_ALIGN;
-    const bool tc_down = ctx->tensor_path_ok && !ctx->force_decode_path && T >= tc_min_tokens_down(ctx->cfg);
-    return launch_combine(ctx, T, ctx->route_k, tc_down ? 1 : ctx->down_splits, out, st);
+    int tc_min[2];
+    step_tc_min(ctx, T, ctx->route_k, tc_min);
+    return launch_combine(ctx, T, ctx->route_k, tc_min[1] > 0 ? ctx->down_splits : 1, tc_min[1], out, st);
+}
+
+// Which experts of a T-token step go to the tensor-core kernels (see Sched::tc_min). Today's rule reproduces the
+// all-or-nothing switch per projection; MIRA_OPT_HYBRID_MIN_UP / _DOWN override it.
+void step_tc_min(const mira_ctx* ctx, int T, int k, int out_min[2]) {
+    (void)k;
+    const bool tc_ok = ctx->tensor_path_ok && !ctx->force_decode_path;
+    out_min[0] = (tc_ok && T >= tc_min_tokens_up(ctx->cfg)) ? 0 : INT_MAX;
+    out_min[1] = (tc_ok && T >= tc_min_tokens_down(ctx->cfg)) ? 0 : INT_MAX;
+    if (tc_ok && T >= kTensorPathMinTokens)
+        for (int p = 0; p < 2; ++p)
+            if (ctx->hybrid_min[p] >= 0) out_min[p] = ctx->hybrid_min[p];
 }
 
 }  // namespace mira
@@ -366,6 +383,10 @@ mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value) {
     if (option == MIRA_OPT_TENSOR_LAYOUT && value >= 0 && value <= 5) { ctx->tc_layout = value; return MIRA_OK; }
     if (option == MIRA_OPT_UP_CONVERSION && value >= 0 && value <= 2) { ctx->up_conversion = value; return MIRA_OK; }
     if (option == MIRA_OPT_TEST_WAIT_TIMEOUT) { ctx->test_wait_timeout = value != 0; return MIRA_OK; }
+    if ((option == MIRA_OPT_HYBRID_MIN_UP || option == MIRA_OPT_HYBRID_MIN_DOWN) && value >= -1) {
+        ctx->hybrid_min[option == MIRA_OPT_HYBRID_MIN_UP ? 0 : 1] = value;
+        return MIRA_OK;
+    }
     return MIRA_ERR_INVALID_ARG;
 }
 

@@ -80,10 +80,12 @@ struct ItemTable {             // the schedule, copied to shared memory once per
 };
 
 __device__ __forceinline__ void load_table(ItemTable& tab, const Sched* __restrict__ sched, int which) {
-    if (threadIdx.x == 0) { tab.n_active = sched->n_active; tab.total_tb = sched->total_tb; }
+    // the token blocks and costs of THIS projection's streaming work: an expert that the tensor-core kernel takes has
+    // none, and the searches below skip such zero-length entries
+    if (threadIdx.x == 0) { tab.n_active = sched->n_active; tab.total_tb = sched->total_tb[which]; }
     for (int i = threadIdx.x; i < kMaxExperts; i += blockDim.x) tab.act_expert[i] = (uint8_t)sched->act_expert[i];
     for (int i = threadIdx.x; i <= kMaxExperts; i += blockDim.x) {
-        tab.tb_prefix[i] = sched->tb_prefix[i];
+        tab.tb_prefix[i] = sched->tb_prefix[which][i];
         tab.w_prefix[i] = sched->w_prefix[which][i];
     }
     __syncthreads();
@@ -586,6 +588,7 @@ struct CombineArgs {
     const int32_t* idx; const float* w; const int32_t* perm; const float* ypart;
     const uint32_t* done_mask; uint32_t* miss_mask; int32_t* status;
     void* out; int T, C, k, ns, E, S, out_fp32; long ypart_stride;
+    const int32_t* count; int down_tc_min;      // terms of experts with count >= down_tc_min have one slice (tensor-core down kernel)
 };
 
 constexpr int kCombineThreads = 128;
@@ -593,6 +596,7 @@ constexpr int kCombineMaxTerms = kMaxTopK + 16;     // routed choices + shared e
 
 __global__ void __launch_bounds__(kCombineThreads) k_combine(CombineArgs A) {
     __shared__ int s_pos[kCombineMaxTerms];
+    __shared__ int s_S[kCombineMaxTerms];
     __shared__ float s_w[kCombineMaxTerms];
     const int t = blockIdx.y;
     const int c = (blockIdx.x * kCombineThreads + threadIdx.x) * 4;
@@ -606,6 +610,7 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine(CombineArgs A) {
         const bool done = (A.done_mask[e >> 5] >> (e & 31)) & 1u;
         if (!done && blockIdx.x == 0) { atomicOr(A.miss_mask + (e >> 5), 1u << (e & 31)); atomicOr(A.status, 1); }
         s_pos[j] = done ? pos : -1;
+        s_S[j] = (A.count[e] >= A.down_tc_min) ? 1 : A.S;
         s_w[j] = wj;
     }
     pdl_wait();            // the routing results above are older than the kernel before this one; the partial sums are not
@@ -637,10 +642,11 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine(CombineArgs A) {
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj) {
                 const int pos = (j0 + jj < kk) ? s_pos[j0 + jj] : -1;
+                const int Sj = (j0 + jj < kk) ? s_S[j0 + jj] : 0;
                 const float* yp = A.ypart + (size_t)max(pos, 0) * A.C + c;
 #pragma unroll
                 for (int s = 0; s < 8; ++s)
-                    v[jj][s] = (pos >= 0 && s0 + s < A.S)
+                    v[jj][s] = (pos >= 0 && s0 + s < Sj)
                         ? __ldcs(reinterpret_cast<const float4*>(yp + (size_t)(s0 + s) * A.ypart_stride))
                         : make_float4(0.f, 0.f, 0.f, 0.f);
             }
@@ -706,7 +712,7 @@ mira_status launch_down(mira_ctx* ctx, void* const* slots, const int32_t* slot_m
     return MIRA_OK;
 }
 
-mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, void* out, cudaStream_t st) {
+mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, int down_tc_min, void* out, cudaStream_t st) {
     CombineArgs A;
     A.idx = ws_ptr<int32_t>(ctx, ctx->lay.idx); A.w = ws_ptr<float>(ctx, ctx->lay.w);
     A.perm = ws_ptr<int32_t>(ctx, ctx->lay.perm); A.ypart = ws_ptr<float>(ctx, ctx->lay.ypart);
@@ -715,6 +721,7 @@ mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, void* out, c
     A.done_mask = A.miss_mask + 8;
     A.out = out; A.T = T; A.C = ctx->cfg.hidden; A.k = k; A.ns = ctx->cfg.n_shared; A.E = ctx->cfg.n_experts;
     A.S = splits; A.out_fp32 = ctx->cfg.out_dtype;
+    A.count = ws_ptr<int32_t>(ctx, ctx->lay.count); A.down_tc_min = down_tc_min;
     A.ypart_stride = (long)T * (k + ctx->cfg.n_shared) * ctx->cfg.hidden;
     dim3 grid((ctx->cfg.hidden / 4 + kCombineThreads - 1) / kCombineThreads, T);
     ProfScope ps(ctx, MIRA_K_COMBINE, st);

@@ -290,9 +290,10 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     if (tid == 0) {
         int acc = 0;
         // S5 of a wide-range expert holds both windows of a token in one tile: half as many tokens per tile
+        const int tc_min = A.sched->tc_min[DOWN ? 1 : 0];      // hybrid step: experts with fewer pairs belong to the streaming kernel
         for (int a = 0; a < n_active; ++a) {
             const int tn = (DOWN && s_wide[a]) ? kTileN / 2 : kTileN;
-            s_ntile[a] = acc; acc += (s_cnt[a] + tn - 1) / tn;
+            s_ntile[a] = acc; acc += s_cnt[a] >= tc_min ? (s_cnt[a] + tn - 1) / tn : 0;
         }
         s_ntile[n_active] = acc;
     }
@@ -692,9 +693,10 @@ k_ffn_tc_pair(TcArgs A, const __grid_constant__ HalfMaps bmaps, const __grid_con
     __syncthreads();
     if (tid == 0) {
         int acc = 0;
+        const int tc_min = A.sched->tc_min[DOWN ? 1 : 0];
         for (int a = 0; a < n_active; ++a) {
             const int tn = (DOWN && s_wide[a]) ? kPairTileN / 2 : kPairTileN;
-            s_ntile[a] = acc; acc += (s_cnt[a] + tn - 1) / tn;
+            s_ntile[a] = acc; acc += s_cnt[a] >= tc_min ? (s_cnt[a] + tn - 1) / tn : 0;
         }
         s_ntile[n_active] = acc;
     }
@@ -963,7 +965,7 @@ k_ffn_tc_pair(TcArgs A, const __grid_constant__ HalfMaps bmaps, const __grid_con
 struct GatherArgs {
     const __half* x16; const int32_t* row_token; __half* x16p; const int32_t* offset; void* const* slots;
     const int32_t* slot_map; const float* xscale; const float* xnorm; const float* xsum; float* xs_pos; float* hm_pos;
-    float* sum_pos; float* hscale; const int32_t* hexp;
+    float* sum_pos; float* hscale; const int32_t* hexp; const Sched* sched;
     int C, R, Etot;
 };
 
@@ -972,12 +974,13 @@ __global__ void __launch_bounds__(128) k_gather_x16p(GatherArgs G) {
     pdl_wait();            // the routing kernels' results; see launch_pdl
     pdl_launch();
     const int pos = blockIdx.x, tok = G.row_token[pos];
-    const uint4* src = reinterpret_cast<const uint4*>(G.x16 + (size_t)tok * G.C);
-    uint4* dst = reinterpret_cast<uint4*>(G.x16p + (size_t)pos * G.C);
-    for (int i = threadIdx.x; i < G.C / 8; i += 128) dst[i] = src[i];
     for (int e = threadIdx.x; e < G.Etot; e += 128)
         if (G.offset[e] <= pos && pos < G.offset[e + 1]) s_e = e;
     __syncthreads();
+    if (G.offset[s_e + 1] - G.offset[s_e] < G.sched->tc_min[0]) return;     // hybrid step: this expert's up/gate is the streaming kernel's
+    const uint4* src = reinterpret_cast<const uint4*>(G.x16 + (size_t)tok * G.C);
+    uint4* dst = reinterpret_cast<uint4*>(G.x16p + (size_t)pos * G.C);
+    for (int i = threadIdx.x; i < G.C / 8; i += 128) dst[i] = src[i];
     if (threadIdx.x == 0) {
         if (G.slot_map[s_e] < 0) return;                        // expert not resident: its pairs are skipped everywhere
         const int f = max(-120, min(120, -(G.hexp[s_e] + 11 + 2 * expo_f(G.xnorm[tok]))));
@@ -1118,7 +1121,7 @@ mira_status launch_up_gate_tc(mira_ctx* ctx, void* const* slots, const int32_t* 
     G.xscale = ws_ptr<float>(ctx, ctx->lay.xscale); G.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm);
     G.xs_pos = ws_ptr<float>(ctx, ctx->lay.xs_pos); G.hm_pos = ws_ptr<float>(ctx, ctx->lay.hm_pos);
     G.sum_pos = ws_ptr<float>(ctx, ctx->lay.sum_pos); G.xsum = ws_ptr<float>(ctx, ctx->lay.xsum);
-    G.hscale = ws_ptr<float>(ctx, ctx->lay.hscale); G.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
+    G.hscale = ws_ptr<float>(ctx, ctx->lay.hscale); G.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp); G.sched = A.sched;
     G.C = ctx->cfg.hidden; G.R = ctx->cfg.ffn; G.Etot = Et(ctx->cfg);
     if (ctx->test_wait_timeout) {          // one launch whose waits run out (MIRA_OPT_TEST_WAIT_TIMEOUT)
         A.spin_limit = 1u << 12;

@@ -24,9 +24,14 @@ constexpr int kLoShift = 24;
 // Device-resident schedule written by the grouping kernel and read by the expert kernels.
 struct Sched {
     int32_t n_active;                  // experts with at least one pair AND a resident slot
-    int32_t total_tb;                  // token blocks over all active experts
     int32_t act_expert[kMaxExperts];   // active expert ids, ascending
-    int32_t tb_prefix[kMaxExperts + 1];// exclusive prefix sum of token blocks per active expert
+    // A step may split its experts between the two kernel families ("hybrid" step): an active expert with fewer than
+    // tc_min[p] pairs is taken by the weight-streaming kernel of projection p (0 up/gate, 1 down), the others by
+    // the tcgen05 kernel (tc_min = 0: all tensor-core; INT_MAX: all streaming). The streaming kernels' work lists:
+    int32_t tc_min[2];
+    int32_t total_tb[2];               // token blocks of the streaming kernel of projection p
+    int32_t tb_prefix[2][kMaxExperts + 1];   // exclusive prefix sum of those token blocks per active expert (0 blocks for
+                                             // an expert the tensor-core kernel takes)
     // Exclusive prefix sums of the COST of the token blocks, [0] for the up/gate kernel, [1] for the down kernel.
     // A block of 1-8, 9-16, 17-24, 25-32 tokens costs block_cost(., 1..4): the streaming kernels split the work
     // between CTAs by cost, not by block count. Alone, a full block takes about 1.5x the time of an 8-token block
@@ -112,6 +117,8 @@ struct mira_ctx {
     bool force_decode_path = false;
     int tc_layout = 0;                 // 0: chosen per step; 1..3 force a tile layout of the tensor-core kernels (MIRA_OPT_TENSOR_LAYOUT)
     bool test_wait_timeout = false;    // the next tcgen05 up/gate launch drops one load and shortens its waits (MIRA_OPT_TEST_WAIT_TIMEOUT)
+    int hybrid_min[2] = {-1, -1};      // MIRA_OPT_HYBRID_MIN_UP / _DOWN: -1 = chosen per step, else the pair count from which an
+                                       // expert goes to the tcgen05 kernel of that projection (0: all, INT_MAX: none)
     int up_conversion = 0;             // 0: chosen per batch on the device; 1: exact; 2: offset subnormals (MIRA_OPT_UP_CONVERSION)
     bool prof_on = false;
     size_t prof_used = 0;
@@ -152,6 +159,7 @@ mira_status launch_unpack(mira_ctx*, const void* blob, int8_t* q1, int8_t* q2, i
 // route.cu
 mira_status launch_scores(mira_ctx*, const void* x, int T, const void* w, const float* b, int E,
                           float* scores, __half* x16, float* xscale, float* xnorm, cudaStream_t);
+// (launch_route and launch_schedule write the schedule for the thresholds step_tc_min gives for (T, k))
 mira_status launch_route(mira_ctx*, const void* x, int T, const void* w, const float* b, int k,
                          const RouteView& rv, __half* x16, float* xscale, float* xnorm, void* const* slots,
                          const int32_t* slot_map, int* fused_schedule, cudaStream_t, bool quiet_schedule = false);
@@ -162,7 +170,7 @@ mira_status launch_pool(mira_ctx*, const float* token_scores, int T, int E, floa
 // expert_ffn.cu
 mira_status launch_up_gate(mira_ctx*, void* const* slots, const int32_t* slot_map, cudaStream_t);
 mira_status launch_down(mira_ctx*, void* const* slots, const int32_t* slot_map, cudaStream_t);
-mira_status launch_combine(mira_ctx*, int T, int k, int splits, void* out, cudaStream_t);
+mira_status launch_combine(mira_ctx*, int T, int k, int splits, int down_tc_min, void* out, cudaStream_t);
 // expert_ffn_tc.cu (tcgen05 path for prefill-sized batches)
 bool tc_shape_ok(const mira_config&);
 bool build_tensor_maps(mira_ctx*);
@@ -178,6 +186,9 @@ mira_status set_tc_attributes();
 constexpr int kTensorPathMinTokens = 16;    // below, no buffers of the tensor path are laid out
 inline int tc_min_tokens_up(const mira_config& c) { return c.n_experts + c.n_shared > 16 ? 32 : 56; }
 inline int tc_min_tokens_down(const mira_config& c) { return c.n_experts + c.n_shared > 16 ? 16 : 40; }
+// Per projection (0 up/gate, 1 down): the pair count from which an expert of a T-token step goes to the tcgen05
+// kernel (0: every expert; INT_MAX: none). The same rule for every wave of a routed batch.
+void step_tc_min(const mira_ctx* ctx, int T, int k, int out_min[2]);
 mira_status set_route_attributes();
 // mixture_head.cu
 mira_status launch_mixture(mira_ctx*, const void* hidden, int T, const float* logits, const int32_t* count, int k_top,

@@ -343,6 +343,7 @@ struct SchedArgs {
     //   dc_heavy whether some token's activations have a sum so large against their norm that the up/gate kernels
     //            must convert the codes exactly instead of through offset subnormals (see dc_heavy_tokens).
     void* const* slots; int32_t* hexp; const float* xsum; const float* xnorm; const float* xscale;
+    int tc_min[2];                      // hybrid thresholds of the step (see Sched)
     int T, R, C, per_matrix, n_main;    // n_main: CTAs of the launch that are not statistics CTAs
 };
 
@@ -417,24 +418,27 @@ __device__ __forceinline__ void expert_stats(const SchedArgs& S, int e) {
 
 // Serial tail of the schedule (one thread): the active experts in ascending order with the prefix sums of their
 // token blocks and of the blocks' costs. tb[i] = token blocks of expert i if it is active, else 0.
-__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot, int dc_heavy) {
-    int n = 0, a = 0, wu = 0, wd = 0;
+__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot, int dc_heavy,
+                                               int min_up, int min_down) {
+    int n = 0, au = 0, ad = 0, wu = 0, wd = 0;
     sched->dc_heavy = dc_heavy;
+    sched->tc_min[0] = min_up; sched->tc_min[1] = min_down;
     for (int i = 0; i < Etot; ++i) {
         const int b = tb[i];
         if (b > 0) {
-            sched->act_expert[n] = i; sched->tb_prefix[n] = a;
+            sched->act_expert[n] = i;
+            sched->tb_prefix[0][n] = au; sched->tb_prefix[1][n] = ad;
             sched->w_prefix[0][n] = wu; sched->w_prefix[1][n] = wd;
             const int last = (count[i] - (b - 1) * kTokBlock + 7) >> 3;          // n-tiles of the last block, 1..4
-            wu += (b - 1) * block_cost(0, 4) + block_cost(0, last);
-            wd += (b - 1) * block_cost(1, 4) + block_cost(1, last);
-            a += b; ++n;
+            if (count[i] < min_up) { wu += (b - 1) * block_cost(0, 4) + block_cost(0, last); au += b; }      // streaming up/gate
+            if (count[i] < min_down) { wd += (b - 1) * block_cost(1, 4) + block_cost(1, last); ad += b; }    // streaming down
+            ++n;
         }
     }
-    sched->tb_prefix[n] = a;
+    sched->tb_prefix[0][n] = au; sched->tb_prefix[1][n] = ad;
     sched->w_prefix[0][n] = wu; sched->w_prefix[1][n] = wd;
     sched->n_active = n;
-    sched->total_tb = a;
+    sched->total_tb[0] = au; sched->total_tb[1] = ad;
 }
 
 // Called by every thread of a CTA of at least kMaxExperts threads. Thread e looks at expert e; a warp covers one word
@@ -460,7 +464,7 @@ __device__ __forceinline__ void schedule_body(const SchedArgs& S, const int* cou
         }
     }
     const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, heavy);    // s_tb is 0 for inactive experts
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, heavy, S.tc_min[0], S.tc_min[1]);    // s_tb is 0 for inactive experts
 }
 
 // S3 for large batches, one CTA; with do_sched also the work schedule of a call that runs every routed expert.
@@ -792,7 +796,7 @@ __global__ void __launch_bounds__(kSingleCtaThreads) k_route_small(TokenArgs A, 
         }
     }
     const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot, heavy);
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot, heavy, S.tc_min[0], S.tc_min[1]);
 }
 
 // S7 pooling: pooled[e] = mean_t score[t][e]; then the k_pred best pooled scores.
@@ -938,13 +942,14 @@ GroupArgs group_args(mira_ctx* ctx, int T, int k, const RouteView& rv) {
     G.host_count = ctx->notify_count; G.host_flag = ctx->notify_flag; G.host_seq = ctx->notify_seq;
     return G;
 }
-SchedArgs sched_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map, const uint32_t* host_mask, int T, int n_main,
+SchedArgs sched_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map, const uint32_t* host_mask, int T, int k, int n_main,
                      bool quiet = false) {
     SchedArgs S;
     S.quiet = quiet ? 1 : 0;
     S.slots = slots; S.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
     S.xsum = ws_ptr<float>(ctx, ctx->lay.xsum); S.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm); S.xscale = ws_ptr<float>(ctx, ctx->lay.xscale);
     S.T = T; S.R = ctx->cfg.ffn; S.C = ctx->cfg.hidden; S.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX; S.n_main = n_main;
+    step_tc_min(ctx, T, k, S.tc_min);
     const int Etot = Et(ctx->cfg);
     for (int i = 0; i < 8; ++i) S.mask.w[i] = (host_mask == nullptr) ? 0xffffffffu : (i < (Etot + 31) / 32 ? host_mask[i] : 0u);
     S.slot_map = slot_map;
@@ -974,7 +979,7 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
         A.k = k; A.idx = rv.idx; A.wts = rv.w;
         A.ticket = ws_ptr<unsigned>(ctx, ctx->lay.status) + 8;
         A.do_sched = slot_map != nullptr;
-        SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, single ? 1 : T, quiet_schedule);
+        SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, k, single ? 1 : T, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_ROUTE, st);
         if (single) MIRA_CUDA_OK(launch_pdl(k_route_small, dim3(1 + n_stat), dim3(kSingleCtaThreads), (size_t)T * C * 2, st, A, G, S));
         else MIRA_CUDA_OK(launch_pdl(k_route_token, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
@@ -996,7 +1001,7 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
     {
         // the schedule of a run over all experts comes out of the same launch
         const int do_sched = slot_map != nullptr;
-        SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, 1, quiet_schedule);
+        SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, k, 1, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_GROUP, st);
         k_group<<<1 + n_stat, 1024, 0, st>>>(G, S, do_sched);
         if (fused_schedule) *fused_schedule = do_sched;
@@ -1008,7 +1013,7 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
 
 mira_status launch_schedule(mira_ctx* ctx, int T, void* const* slots, const int32_t* slot_map, const uint32_t* host_mask,
                             int all_experts, cudaStream_t st) {
-    SchedArgs S = sched_args(ctx, slots, slot_map, all_experts ? nullptr : host_mask, T, 1);
+    SchedArgs S = sched_args(ctx, slots, slot_map, all_experts ? nullptr : host_mask, T, ctx->route_k, 1);
     ProfScope ps(ctx, MIRA_K_SCHEDULE, st);
     k_schedule<<<1 + (slots != nullptr ? Et(ctx->cfg) : 0), 256, 0, st>>>(ws_ptr<int32_t>(ctx, ctx->lay.count), Et(ctx->cfg), S);
     ctx->launches += 1;

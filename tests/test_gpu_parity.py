@@ -487,3 +487,26 @@ def test_quantizer_does_not_depend_on_the_token_capacity():
     out = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k)
     res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k, n_shared=sh.n_shared)
     assert gate_a(out.cpu().numpy(), res["out64"]) <= TOL
+
+
+@pytest.mark.parametrize("mins", [(9, 9), (17, 2 ** 31 - 1), (2 ** 31 - 1, 5), (5, 17), (33, 33), (1, 1)])
+@pytest.mark.parametrize("shape", ["tiny", "small_shared"])
+def test_hybrid_steps_split_the_experts_between_the_kernel_families(shape, mins):
+    """A step may hand the experts with few pairs to the weight-streaming kernels and the others to the tcgen05
+    kernels, per projection (thresholds forced here; the skewed routing gives both kinds in every batch). Against the
+    oracle, and as waves (the split is a property of the step, so waves reproduce the single call bit for bit)."""
+    sh = inputs.TINY if shape == "tiny" else SMALL_SHARED
+    for T in (40, 130):
+        wl, d, m, blobs, slots, slot_map = _setup(sh, T, out_fp32=True)
+        m.hybrid_min(*mins)
+        out, dbg = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k, debug=True)
+        torch.cuda.synchronize()
+        assert m.poll_status()[0] == 0
+        cnt = dbg["count"].cpu().numpy()
+        res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k, n_shared=sh.n_shared)
+        assert gate_a(out.cpu().numpy(), res["out64"]) <= TOL, f"T={T} mins={mins} counts={cnt.tolist()}"
+        needed = [e for e, c in enumerate(cnt.tolist()) if c > 0]
+        m.route(d["x"], d["wr"], d["bias"], sh.k)
+        m.moe_experts(d["x"], slots, slot_map, expert_ids=needed[::2], final_wave=False)
+        two = m.moe_experts(d["x"], slots, slot_map, expert_ids=needed[1::2], final_wave=True)
+        assert torch.equal(out, two)
