@@ -55,13 +55,14 @@ constexpr int kWStage = 4 * kWWarp;  // the four warps of a converter group
 //   ISSUERS MMA-issuing warps (2: they take the K-blocks in turn, so one thread's barrier waits and commit overlap
 //           the other's MMAs; a turn barrier keeps the MMAs of a tile in K order)
 // TMEM columns of one CTA: ACC * TN + 32 NS, a power of two, CTAS of them in the SM's 512.
-template <int TN, int NS, int GROUPS, int ACC, int CTAS, int ISSUERS = 1> struct TileCfg {
+template <int TN, int NS, int GROUPS, int ACC, int CTAS, int ISSUERS = 1, int WST = kWStages> struct TileCfg {
     static constexpr int kTileN = TN, kStages = NS, kGroups = GROUPS, kAccBufs = ACC, kCtasPerSm = CTAS, kIssuers = ISSUERS;
+    static constexpr int kWRing = WST;           // depth of each converter group's int8 weight ring (cp.async stages)
     static constexpr int kEpiWarp0 = 4 * GROUPS, kTmaWarp = kEpiWarp0 + 4, kMmaWarp = kEpiWarp0 + 5;
     static constexpr int kThreads = (kMmaWarp + ISSUERS) * 32;
     static constexpr uint32_t kTmemCols = ACC * TN + NS * 32;
     static constexpr int kBTileBytes = TN * kKB * 2;
-    static constexpr size_t kSmem = (size_t)NS * kBTileBytes + (size_t)GROUPS * kWStages * kWStage + 1024;
+    static constexpr size_t kSmem = (size_t)NS * kBTileBytes + (size_t)GROUPS * WST * kWStage + 1024;
     static_assert(kTmemCols == 256 || kTmemCols == 512, "TMEM allocations are powers of two");
     static_assert(kTmemCols * CTAS <= 512, "TMEM has 512 columns per SM");
     static_assert((kSmem + 8 * 1024) * CTAS <= 227 * 1024, "shared memory per SM");
@@ -75,6 +76,10 @@ template <int TN, int NS, int GROUPS, int ACC, int CTAS, int ISSUERS = 1> struct
 using BigTile = TileCfg<192, 4, 2, 2, 1, 2>;    // one CTA per SM, two converter groups, two accumulators, two issuers
 using WideTile = TileCfg<192, 2, 1, 1, 2>;      // two CTAs per SM
 using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
+// (Tried for batches with few tokens per expert and dropped: 64-token tiles with a weight ring of 7 stages instead of
+// 4, and the same tiles with two converter groups per CTA -- 4 groups per SM, 72 registers per thread: Mixtral shape, 64
+// tokens, up/gate 228 and 217 against 226 us; fine-grained 1024 tokens 237 and 239 against 215 us. Neither the weight
+// bytes in flight nor the converters' throughput is what sets the K-block period.)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
 
@@ -233,7 +238,7 @@ __device__ __forceinline__ void convert_row(unsigned (&f)[32], uint32_t saddr) {
 template <bool DOWN, typename TC>
 __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs A, const __grid_constant__ TileMaps bmaps, const __grid_constant__ TileMaps bmaps_lo) {
     constexpr int kTileN = TC::kTileN, kAStages = TC::kStages, kBStages = TC::kStages, kBTileBytes = TC::kBTileBytes;
-    constexpr int kGroups = TC::kGroups, kAccBufs = TC::kAccBufs;
+    constexpr int kGroups = TC::kGroups, kAccBufs = TC::kAccBufs, kWRing = TC::kWRing;
     constexpr int kEpiWarp0 = TC::kEpiWarp0, kTmaWarp = TC::kTmaWarp, kMmaWarp = TC::kMmaWarp, kIssuers = TC::kIssuers;
     constexpr uint32_t kTmemCols = TC::kTmemCols;
     constexpr uint32_t kTmemA = kAccBufs * kTileN;      // first column of the A ring
@@ -331,7 +336,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     if (warp < kEpiWarp0) {
         // ------------------------------------------------ converters: group (warp >> 2) takes the blocks with g % kGroups == group
         const int group = warp >> 2, gw = warp & 3, row = gw * 32 + lane;     // MMA row of this thread
-        const uint32_t w_g = w_s + group * (kWStages * kWStage) + gw * kWWarp;
+        const uint32_t w_g = w_s + group * (kWRing * kWStage) + gw * kWWarp;
         const uint32_t w_cp = w_g + (lane & 7) * kWRow + (lane >> 3) * 16;   // + stage * kWStage + i * 8 * kWRow
         const uint32_t w_rd = w_g + lane * kWRow;                             // + stage * kWStage + q * 16
         uint32_t gbase = 0;                                                   // K-blocks of this CTA's earlier tiles
@@ -350,7 +355,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
             const int kb0 = (int)(((uint32_t)group + kGroups - gbase % kGroups) % kGroups);   // first K-block of this tile that belongs to the group
             const int nmine = (nkb - kb0 + kGroups - 1) / kGroups;                               // its blocks: kb0, kb0 + kGroups, ...
 #pragma unroll
-            for (int s = 0; s < kWStages - 1; ++s) {
+            for (int s = 0; s < kWRing - 1; ++s) {
                 if (s < nmine) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) cp_async16_s(w_cp + s * kWStage + i * 8 * kWRow, src + i * src_step + (size_t)(kb0 + kGroups * s) * kKB);
@@ -359,16 +364,16 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
             }
             bool ok = true;
             for (int j = 0; j < nmine; ++j) {
-                const int pre = j + kWStages - 1;
+                const int pre = j + kWRing - 1;
                 if (pre < nmine) {
-                    const int ws = pre % kWStages;
+                    const int ws = pre % kWRing;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) cp_async16_s(w_cp + ws * kWStage + i * 8 * kWRow, src + i * src_step + (size_t)(kb0 + kGroups * pre) * kKB);
                 }
                 cp_async_commit();
-                cp_async_wait<kWStages - 1>();
+                cp_async_wait<kWRing - 1>();
                 __syncwarp();                                     // the other lanes' copies of this stage have landed too
-                const int ws = j % kWStages;
+                const int ws = j % kWRing;
                 unsigned f[32];                                   // 64 codes as fp16, in k order
                 if (sub) convert_row<true>(f, w_rd + ws * kWStage);
                 else convert_row<false>(f, w_rd + ws * kWStage);
@@ -1106,7 +1111,7 @@ static void launch_tc(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps
         if (DOWN) layout = 0.9 * down_cost(ctx, NarrowTile::kTileN, 1.0) <= down_cost(ctx, WideTile::kTileN, 1.3) ? 1 : 2;
         else layout = avg < kWideMinPerExpert ? 1 : (avg >= 256 && ctx->cfg.n_experts <= 16) ? 3 : 2;
     }
-    if (layout >= 4 && !pair_shape_ok(ctx->cfg)) layout = DOWN ? 2 : 3;
+    if ((layout == 4 || layout == 5) && !pair_shape_ok(ctx->cfg)) layout = DOWN ? 2 : 3;
     if (layout >= 4) launch_pair<DOWN>(ctx, A, st);
     else if (layout == 1) launch_cfg<DOWN, NarrowTile>(ctx, A, maps, st);
     else if (layout == 3) launch_cfg<DOWN, BigTile>(ctx, A, maps, st);
