@@ -1108,7 +1108,9 @@ static void launch_tc(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps
     int layout = ctx->tc_layout;                          // 0 unless a layout is forced (MIRA_OPT_TENSOR_LAYOUT)
     if (layout == 0) {
         // wide only when the estimate is clearly lower: near a tie the narrow layout is the safer one (1536 tokens: 429 / 460)
-        if (DOWN) layout = 0.9 * down_cost(ctx, NarrowTile::kTileN, 1.0) <= down_cost(ctx, WideTile::kTileN, 1.3) ? 1 : 2;
+        // (with fewer than half a narrow tile of tokens per expert on average no expert fills a wide tile: narrow.
+        // Fine-grained layer, 128 tokens: 39 against 45 us)
+        if (DOWN) layout = (2 * avg < NarrowTile::kTileN || 0.9 * down_cost(ctx, NarrowTile::kTileN, 1.0) <= down_cost(ctx, WideTile::kTileN, 1.3)) ? 1 : 2;
         else layout = avg < kWideMinPerExpert ? 1 : (avg >= 256 && ctx->cfg.n_experts <= 16) ? 3 : 2;
     }
     if ((layout == 4 || layout == 5) && !pair_shape_ok(ctx->cfg)) layout = DOWN ? 2 : 3;
