@@ -260,10 +260,12 @@ mira_status mira_predict_mixture(mira_ctx* ctx, int32_t layer, const void* hidde
  * two-SM kernel (tcgen05 cta_group::2: tiles of 256 MMA rows over a cluster of two CTAs, 192 tokens x 4 ring stages
  * or 128 tokens x 8; needs ffn % 128 == 0 and hidden % 256 == 0, else the one-CTA layouts run), for tests and
  * tuning. MIRA_OPT_UP_CONVERSION (value 0..2): how the tcgen05 up/gate kernel turns int8 codes into fp16 operands
- * (the weight-streaming kernels always convert exactly). 0 (the default) decides per batch on the device: codes go in
- * as (code + 128) * 2^-24 with the offset taken out afterwards, unless some token's activations have a sum so large
- * against their norm (hidden size * |sum x| > 24576 * |x|_2) that the subtraction would cost accuracy, in which case
- * the codes are converted exactly; 1 forces the exact conversion, 2 the offset form (tests and tuning). MIRA_OPT_TEST_WAIT_TIMEOUT (value 1; test hook): the next tcgen05
+ * (the weight-streaming kernels always convert exactly). 0 and 1: exactly (the default). 2: as (code + 128) * 2^-24 with
+ * the offset 128 * sum(x) taken out afterwards, 1.6 % faster at 2048 tokens; only accurate while the activations of every
+ * token are close to zero-mean and every row's codes are well spread (the subtraction costs about
+ * hidden size * |sum x| / (32 |x|_2) * 2^-27 relative to a row of typical codes, more for rows of small codes), which
+ * the library does not check; tiles of wide-range experts convert exactly regardless.
+ * MIRA_OPT_TEST_WAIT_TIMEOUT (value 1; test hook): the next tcgen05
  * up/gate launch of this context leaves out one activation load in its first CTA and gives up its waits after 4096
  * polls instead of 2^24, so that CTA takes the time-out path (status MIRA_ERR_TIMEOUT at the next poll); the option
  * clears itself with that launch. MIRA_OPT_HYBRID_MIN_UP / MIRA_OPT_HYBRID_MIN_DOWN (value >= -1): a step may split its

@@ -343,7 +343,7 @@ class Mira:
         _check(mira_set_option(self._ctx, MIRA_OPT_TENSOR_LAYOUT, int(layout)), "mira_set_option")
 
     def up_conversion(self, mode: int) -> None:
-        """0: decided per batch on the device (default); 1: exact code conversion in the up/gate kernels; 2: offset subnormals."""
+        """tcgen05 up/gate kernel: 0, 1: exact code conversion (default); 2: offset subnormals (faster, input-dependent accuracy)."""
         _check(mira_set_option(self._ctx, MIRA_OPT_UP_CONVERSION, int(mode)), "mira_set_option")
 
     def hybrid_min(self, up: int = -1, down: int = -1) -> None:

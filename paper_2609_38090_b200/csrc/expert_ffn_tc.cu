@@ -96,7 +96,7 @@ struct TcArgs {
     int32_t* status;
     int R, C, act_on_w1;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
-    int up_conversion;          // up/gate codes: 0 as the schedule's dc_heavy flag says, 1 exact, 2 offset subnormals
+    int up_conversion;          // up/gate codes: 0, 1 exact conversion; 2 offset subnormals
     uint32_t spin_limit;        // polls after which a barrier wait gives up (kSpinLimit; shortened by MIRA_OPT_TEST_WAIT_TIMEOUT)
     int drop_first_load;        // test hook: CTA 0 leaves out the activation load of its first K-block, so the waits on that
                                 // stage run out and the kernel leaves through its time-out path
@@ -184,14 +184,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const unsigned (&v)[32
     asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
 }
 
-// The up/gate kernel may feed the codes as fp16 subnormals (code + 128) * 2^-24 and undo offset and scale in its
-// epilogue with the per-token sum of the activations: two fewer instructions per four weights in the converters.
-// The subtracted term grows with the sum of a token's activations, so batches that hold a token whose sum is large
-// against its norm (the schedule's dc_heavy flag) take the exact conversion, as the down kernel always does. So do
-// the tiles of wide-range experts: the offset is 128 per code whatever the code, so rows whose codes are small
-// (a row triple whose scale is set by one large weight or by another matrix's row) lose the bits the offset takes
-// (measured: 1e-2 on a layer whose gate codes are mostly 0 and +-1).
-
+// The up/gate kernel can feed the codes as fp16 subnormals (code + 128) * 2^-24 and undo offset and scale in its
+// epilogue with the per-token sum of the activations: two fewer instructions per four weights in the converters
+// (1.6 % of the kernel at 2048 tokens). It is an option, not the default (MIRA_OPT_UP_CONVERSION = 2): the tensor
+// cores add in fp32 with truncation, so the subtracted term 128 * sum(x) costs accuracy in proportion to
+// |sum x| / (rms of the row's codes * |x|_2) and to the hidden size. With Gaussian weights and zero-mean activations
+// that is invisible up to a hidden size of about 8000; a mean of the order of the spread costs 6e-3 at 4096, and a
+// row triple whose scale is set by another matrix's row (codes of a few units) fails at a mean of 0.3 even at 512.
+// Neither can be seen from the scales, so the default converts exactly. The tiles of wide-range experts always do.
 __device__ __forceinline__ unsigned cvt_exact_lo(unsigned u) {      // bytes 0,1 of (code + 128) -> half2 of codes
     unsigned v = __byte_perm(u, 0x64646464u, 0x4140);
     __half2 r = __hsub2(*reinterpret_cast<__half2*>(&v), __half2half2(__ushort_as_half(0x6480)));
@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 
     // per-expert table: one round of parallel loads, then a serial prefix over shared memory
     const int n_active = A.sched->n_active;
-    const bool sub_batch = !DOWN && (A.up_conversion == 2 || (A.up_conversion == 0 && A.sched->dc_heavy == 0));
+    const bool sub_batch = !DOWN && A.up_conversion == 2;
     if (tid < kMaxExperts && tid < n_active) {
         const int e = A.sched->act_expert[tid];
         s_cnt[tid] = A.count[e];
@@ -676,7 +676,7 @@ k_ffn_tc_pair(TcArgs A, const __grid_constant__ HalfMaps bmaps, const __grid_con
     auto turn = [&](int q) { return bar0 + 8u * (2 * kPairStages + 4 + q); };
 
     const int n_active = A.sched->n_active;
-    const bool sub_batch = !DOWN && (A.up_conversion == 2 || (A.up_conversion == 0 && A.sched->dc_heavy == 0));
+    const bool sub_batch = !DOWN && A.up_conversion == 2;
     if (tid < kMaxExperts && tid < n_active) {
         const int e = A.sched->act_expert[tid];
         s_cnt[tid] = A.count[e];

@@ -39,9 +39,6 @@ struct Sched {
     // the gap is wider, because the CTAs of small blocks speed up while the others are compute bound and leave
     // them memory bandwidth, so the costs are those that balanced skewed 16- and 32-token batches best.
     int32_t w_prefix[2][kMaxExperts + 1];
-    // 1 if some token of the batch has activations whose sum is large against their norm: the up/gate kernels then
-    // convert the codes exactly instead of through offset subnormals (see dc_heavy_tokens in route.cu).
-    int32_t dc_heavy;
 };
 __host__ __device__ constexpr int block_cost(int which, int n_tiles) {       // which: 0 up/gate, 1 down; n_tiles 1..4
     return which == 0 ? (n_tiles <= 1 ? 16 : n_tiles == 2 ? 22 : n_tiles == 3 ? 27 : 31)
@@ -119,7 +116,7 @@ struct mira_ctx {
     bool test_wait_timeout = false;    // the next tcgen05 up/gate launch drops one load and shortens its waits (MIRA_OPT_TEST_WAIT_TIMEOUT)
     int hybrid_min[2] = {-1, -1};      // MIRA_OPT_HYBRID_MIN_UP / _DOWN: -1 = chosen per step, else the pair count from which an
                                        // expert goes to the tcgen05 kernel of that projection (0: all, INT_MAX: none)
-    int up_conversion = 0;             // 0: chosen per batch on the device; 1: exact; 2: offset subnormals (MIRA_OPT_UP_CONVERSION)
+    int up_conversion = 0;             // tcgen05 up/gate kernel: 0, 1: exact code conversion; 2: offset subnormals (MIRA_OPT_UP_CONVERSION)
     bool prof_on = false;
     size_t prof_used = 0;
     std::vector<mira::ProfRec> prof;   // per-launch event pairs, reused between reads

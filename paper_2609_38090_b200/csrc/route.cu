@@ -337,32 +337,12 @@ struct MaskArg { uint32_t w[8]; };
 struct SchedArgs {
     const int32_t* slot_map; MaskArg mask; Sched* sched; int32_t* status; uint32_t* miss_mask; uint32_t* done_mask;
     int quiet;      // 1: a routed expert without a slot is left for a later wave, not reported as a miss
-    // Inputs of the two numerical decisions the expert kernels take from the schedule stage:
-    //   hexp[e]  exponent of the largest magnitude the intermediate of expert e is expected to reach per unit of
-    //            |x|^2 (from the largest row scale of the blob in its slot), written by the statistics CTAs below;
-    //   dc_heavy whether some token's activations have a sum so large against their norm that the up/gate kernels
-    //            must convert the codes exactly instead of through offset subnormals (see dc_heavy_tokens).
-    void* const* slots; int32_t* hexp; const float* xsum; const float* xnorm; const float* xscale;
+    // hexp[e]: exponent of the largest magnitude the intermediate of expert e is expected to reach per unit of |x|^2
+    // (from the largest row scale of the blob in its slot), then the wide-range flags; written by the statistics CTAs.
+    void* const* slots; int32_t* hexp;
     int tc_min[2];                      // hybrid thresholds of the step (see Sched)
     int T, R, C, per_matrix, n_main;    // n_main: CTAs of the launch that are not statistics CTAs
 };
-
-// The tcgen05 up/gate kernel may feed the codes as (code + 128) * 2^-24 and subtract 128 * sum(x) afterwards. The tensor
-// cores add in fp32 with truncation, so the subtracted term costs about C / 16 accumulation steps of 2^-24 of ITS
-// size, while the wanted sum is about 32 |x|_2 (codes have an rms near 32): the relative error grows like
-// C * |sum x| / |x|_2 (measured on B200: nothing visible at 11 k, 2e-3 added at 82 k). A batch takes the exact
-// conversion when any of its tokens exceeds the bound below; zero-mean activations (|sum x| a few times |x|_2 at
-// most) stay under it up to a hidden size of about 6000.
-constexpr float kDcBound = 24576.f;     // C * |sum x| / |x|_2 from which the exact conversion is used
-
-// Called by every thread of the CTA that writes the schedule. xsum / xnorm may have been written by other CTAs of
-// the same launch (fence + ticket before this call), hence the L2 loads.
-__device__ __forceinline__ int dc_heavy_tokens(const SchedArgs& S) {
-    int heavy = 0;
-    for (int t = threadIdx.x; t < S.T; t += blockDim.x)
-        heavy |= fabsf(__ldcg(S.xsum + t)) * __ldcg(S.xscale + t) * (float)S.C > kDcBound * __ldcg(S.xnorm + t);   // xsum is in pre-scaled units
-    return __syncthreads_or(heavy);
-}
 
 // Statistics CTA of expert e (every thread of the CTA calls it): the largest row scale of the blob in the expert's
 // slot, as the exponent the SwiGLU epilogues use to place the fp16 intermediate. Shared scale: the intermediate
@@ -418,10 +398,9 @@ __device__ __forceinline__ void expert_stats(const SchedArgs& S, int e) {
 
 // Serial tail of the schedule (one thread): the active experts in ascending order with the prefix sums of their
 // token blocks and of the blocks' costs. tb[i] = token blocks of expert i if it is active, else 0.
-__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot, int dc_heavy,
+__device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, const int* count, int Etot,
                                                int min_up, int min_down) {
     int n = 0, au = 0, ad = 0, wu = 0, wd = 0;
-    sched->dc_heavy = dc_heavy;
     sched->tc_min[0] = min_up; sched->tc_min[1] = min_down;
     for (int i = 0; i < Etot; ++i) {
         const int b = tb[i];
@@ -463,8 +442,8 @@ __device__ __forceinline__ void schedule_body(const SchedArgs& S, const int* cou
             if (miss_w && !S.quiet) { atomicOr(S.miss_mask + (e >> 5), miss_w); atomicOr(S.status, 1); }
         }
     }
-    const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, heavy, S.tc_min[0], S.tc_min[1]);    // s_tb is 0 for inactive experts
+    __syncthreads();
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, S.tc_min[0], S.tc_min[1]);    // s_tb is 0 for inactive experts
 }
 
 // S3 for large batches, one CTA; with do_sched also the work schedule of a call that runs every routed expert.
@@ -795,8 +774,8 @@ __global__ void __launch_bounds__(kSingleCtaThreads) k_route_small(TokenArgs A, 
             if (miss && !S.quiet) { atomicOr(S.miss_mask + (e >> 5), miss); atomicOr(S.status, 1); }
         }
     }
-    const int heavy = dc_heavy_tokens(S);                                 // a barrier for the whole CTA
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot, heavy, S.tc_min[0], S.tc_min[1]);
+    __syncthreads();
+    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, s_count, Etot, S.tc_min[0], S.tc_min[1]);
 }
 
 // S7 pooling: pooled[e] = mean_t score[t][e]; then the k_pred best pooled scores.
@@ -947,7 +926,6 @@ SchedArgs sched_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map,
     SchedArgs S;
     S.quiet = quiet ? 1 : 0;
     S.slots = slots; S.hexp = ws_ptr<int32_t>(ctx, ctx->lay.hexp);
-    S.xsum = ws_ptr<float>(ctx, ctx->lay.xsum); S.xnorm = ws_ptr<float>(ctx, ctx->lay.xnorm); S.xscale = ws_ptr<float>(ctx, ctx->lay.xscale);
     S.T = T; S.R = ctx->cfg.ffn; S.C = ctx->cfg.hidden; S.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX; S.n_main = n_main;
     step_tc_min(ctx, T, k, S.tc_min);
     const int Etot = Et(ctx->cfg);
