@@ -484,6 +484,7 @@ def run_cuda(args):
     if sampler:
         sampler.wait_started()
     layer = ResidentLayer(sh, dev)
+    quantize = dict(layer.quantize)                      # S0 of the headline layer (later layers overwrite the global)
     head = measure_resident(layer, sh.T, args, world, rank, sampler, barrier)
     m, xs = head.pop("_m"), head.pop("_xs")
     wr, bias = layer.wr, layer.bias
@@ -560,8 +561,8 @@ def run_cuda(args):
                         "predictor_note": "device time of mira_predict on one batch: linear head, mean over tokens, top-2 (S7)",
                         "mixture_head_us_per_call": mixture_us,
                         "mixture_head_note": "device time of mira_predict_mixture (ActHead + HistHead + gate) on the routing by-products",
-                        "quantize_ms_per_expert": QUANTIZE_STATS.get("ms_per_expert"),
-                        "quantize_gbs": QUANTIZE_STATS.get("gbs"),
+                        "quantize_ms_per_expert": quantize.get("ms_per_expert"),
+                        "quantize_gbs": quantize.get("gbs"),
                         "quantize_note": "mira_quantize_experts (S0): fp32 W2 read twice, W1 and W3 once, blob written"},
     }
     if others:
