@@ -44,3 +44,18 @@ def test_two_gloo_ranks_reduce_timing_to_the_slowest():
     for r in rows:
         assert r["ms"] == 15.0                                  # max over ranks
         assert abs(r["value"] - 2 * 32 * 4 / 15e-3) < 1e-6      # units of all ranks / slowest time
+
+
+def test_block_statistics_and_traffic_ratio_helpers():
+    """Host logic of bench.py that needs no GPU: the median / best block arithmetic and the lookup of the DRAM-traffic
+    ratio recorded with the ncu capture."""
+    sys.path.insert(0, ROOT)
+    import bench
+    st = bench.block_stats([10.0, 12.0, 11.0, 30.0], steps=20)
+    assert st["blocks"] == 4 and abs(st["ms_per_step"] - 11.5 / 20) < 1e-12 and abs(st["ms_per_step_best"] - 0.5) < 1e-12
+    assert abs(st["timed_seconds"] - 0.063) < 1e-12
+    r = bench.traffic_ratio("k_ffn_up_gate")
+    assert r is not None and 1.0 <= r["ratio"] < 1.1 and r["source"].startswith("profiles/")
+    assert bench.traffic_ratio("no_such_kernel") is None
+    hbm, sustained, burst, src = bench.peaks()
+    assert hbm > 1000 and burst >= sustained > 100 and src in ("measured", "fallback")
