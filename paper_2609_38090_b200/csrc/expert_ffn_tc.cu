@@ -79,7 +79,8 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // (Tried for batches with few tokens per expert and dropped: 64-token tiles with a weight ring of 7 stages instead of
 // 4, and the same tiles with two converter groups per CTA -- 4 groups per SM, 72 registers per thread: Mixtral shape, 64
 // tokens, up/gate 228 and 217 against 226 us; fine-grained 1024 tokens 237 and 239 against 215 us. Neither the weight
-// bytes in flight nor the converters' throughput is what sets the K-block period.)
+// bytes in flight nor the converters' throughput is what sets the K-block period. Three CTAs per SM -- 64-token tiles,
+// two ring stages, 64 registers per thread -- lost 9 to 20 %.)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
 
