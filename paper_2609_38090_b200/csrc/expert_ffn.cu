@@ -49,8 +49,8 @@ __device__ __forceinline__ void mma16816(float (&c)[4], unsigned a0, unsigned a1
 // the tensor cores add in fp32 with truncation, so the subtracted term costs accuracy as soon as a token's
 // activations have a mean: measured 6e-3 instead of 1e-3 at hidden size 4096 with mean = spread. It also needs the
 // token sums in the epilogue. Measured on the Mixtral shape the exact form is as fast at 1 and 8 tokens and 0.5 %
-// slower at 32, so the streaming kernels always convert exactly; the tcgen05 up/gate kernel, where the conversion
-// is on the critical path, keeps the offset form for batches without such a token.)
+// slower at 32, so the streaming kernels always convert exactly; the tcgen05 up/gate kernel keeps the offset form
+// as an option.)
 __device__ __forceinline__ unsigned cvt_exact_lo(unsigned u) {
     unsigned v = __byte_perm(u, 0x64646464u, 0x4140);
     __half2 r = __hsub2(*reinterpret_cast<__half2*>(&v), __half2half2(__ushort_as_half(0x6480)));
