@@ -80,7 +80,10 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // 4, and the same tiles with two converter groups per CTA -- 4 groups per SM, 72 registers per thread: Mixtral shape, 64
 // tokens, up/gate 228 and 217 against 226 us; fine-grained 1024 tokens 237 and 239 against 215 us. Neither the weight
 // bytes in flight nor the converters' throughput is what sets the K-block period. Three CTAs per SM -- 64-token tiles,
-// two ring stages, 64 registers per thread -- lost 9 to 20 %.)
+// two ring stages, 64 registers per thread -- lost 9 to 20 %. Weight copies running ahead across tile boundaries, so
+// that a tile does not start with an empty weight ring: down kernel of the fine-grained layer at 1024 tokens 99 against
+// 102 us, up/gate of the Mixtral shape at 128 tokens 226 against 218 us, nothing elsewhere; the stages already converted
+// cover the restart.)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
 
