@@ -272,9 +272,14 @@ mira_status mira_predict_mixture(mira_ctx* ctx, int32_t layer, const void* hidde
  * experts between the two kernel families per projection: experts routed fewer than `value` pairs run on the
  * weight-streaming kernel, the others on the tcgen05 kernel (0: all tensor-core, INT32_MAX: all streaming, -1: the
  * library's rule for the step's token count, the default). Applies to steps of at least 16 tokens of a context whose
- * shape the tensor-core kernels take; set it before the routing call of the step. */
+ * shape the tensor-core kernels take; set it before the routing call of the step.
+ * MIRA_OPT_DOWN_SLICES (value 0..4): reduction slices of the tcgen05 down kernel (one-CTA layouts). Each slice of
+ * the expert-hidden dimension is a tile of its own and writes its own partial sums, which S6 adds in slice order, so
+ * a batch with few token tiles fills the GPU's CTAs more evenly. 0 (the default): chosen per step from the batch size,
+ * the top-k and the configuration, 1 when a tile layout is forced; 1..4: that many, at most ceil(ffn / 4096) (the
+ * partial-sum slices the workspace holds). Set it before the first wave of a step: every wave must use the same. */
 enum { MIRA_OPT_FORCE_DECODE_PATH = 1, MIRA_OPT_TENSOR_LAYOUT = 2, MIRA_OPT_UP_CONVERSION = 3, MIRA_OPT_TEST_WAIT_TIMEOUT = 4,
-       MIRA_OPT_HYBRID_MIN_UP = 5, MIRA_OPT_HYBRID_MIN_DOWN = 6 };
+       MIRA_OPT_HYBRID_MIN_UP = 5, MIRA_OPT_HYBRID_MIN_DOWN = 6, MIRA_OPT_DOWN_SLICES = 7 };
 mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value);
 
 /* ---------------------------------------------------------------------------------------------------------------

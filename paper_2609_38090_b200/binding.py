@@ -123,6 +123,7 @@ MIRA_OPT_UP_CONVERSION = 3
 MIRA_OPT_TEST_WAIT_TIMEOUT = 4
 MIRA_OPT_HYBRID_MIN_UP = 5
 MIRA_OPT_HYBRID_MIN_DOWN = 6
+MIRA_OPT_DOWN_SLICES = 7
 mira_profile_read = lib.mira_profile_read
 KERNEL_CLASSES = ("route", "group", "schedule", "up_gate", "down", "combine", "scores", "pool", "quantize", "unpack")
 mira_status_string = lib.mira_status_string
@@ -351,6 +352,11 @@ class Mira:
         (-1: the library's rule; 0: all; 2**31 - 1: none). Set before the step's routing call."""
         _check(mira_set_option(self._ctx, MIRA_OPT_HYBRID_MIN_UP, int(up)), "mira_set_option")
         _check(mira_set_option(self._ctx, MIRA_OPT_HYBRID_MIN_DOWN, int(down)), "mira_set_option")
+
+    def down_slices(self, n: int = 0) -> None:
+        """Reduction slices of the tcgen05 down kernel (0: chosen per step; 1..4 forced, at most ceil(ffn / 4096)).
+        Set before the first wave of a step."""
+        _check(mira_set_option(self._ctx, MIRA_OPT_DOWN_SLICES, int(n)), "mira_set_option")
 
     def test_wait_timeout(self) -> None:
         """Test hook: the next tcgen05 up/gate launch takes its time-out path in one CTA (see MIRA_OPT_TEST_WAIT_TIMEOUT)."""

@@ -132,7 +132,8 @@ mira_status do_experts(mira_ctx* ctx, int T, void* const* slots, const int32_t* 
     if (tc_min[0] < INT_MAX && (s = launch_up_gate_tc(ctx, slots, slot_map, st)) != MIRA_OK) return s;
     if (tc_min[1] > 0 && (s = launch_down(ctx, slots, slot_map, st)) != MIRA_OK) return s;
     if (tc_min[1] < INT_MAX && (s = launch_down_tc(ctx, slots, slot_map, st)) != MIRA_OK) return s;
-    if (final_wave) s = launch_combine(ctx, T, ctx->route_k, tc_min[1] > 0 ? ctx->down_splits : 1, tc_min[1], out, st);
+    if (final_wave) s = launch_combine(ctx, T, ctx->route_k, tc_min[1] > 0 ? ctx->down_splits : 1,
+                                       tc_min[1] < INT_MAX ? down_tc_slices(ctx) : 1, tc_min[1], out, st);
     return s;
 }
 
@@ -159,7 +160,8 @@ mira_status combine_only(mira_ctx* ctx, int T, void* out, cudaStream_t st) {
     if (misaligned(out)) return MIRA_ERR_ALIGN;
     int tc_min[2];
     step_tc_min(ctx, T, ctx->route_k, tc_min);
-    return launch_combine(ctx, T, ctx->route_k, tc_min[1] > 0 ? ctx->down_splits : 1, tc_min[1], out, st);
+    return launch_combine(ctx, T, ctx->route_k, tc_min[1] > 0 ? ctx->down_splits : 1,
+                          tc_min[1] < INT_MAX ? down_tc_slices(ctx) : 1, tc_min[1], out, st);
 }
 
 // Which experts of a T-token step go to the tensor-core kernels (see Sched::tc_min). Today's rule reproduces the
@@ -382,6 +384,7 @@ mira_status mira_set_option(mira_ctx* ctx, int32_t option, int32_t value) {
     if (option == MIRA_OPT_FORCE_DECODE_PATH) { ctx->force_decode_path = value != 0; return MIRA_OK; }
     if (option == MIRA_OPT_TENSOR_LAYOUT && value >= 0 && value <= 5) { ctx->tc_layout = value; return MIRA_OK; }
     if (option == MIRA_OPT_UP_CONVERSION && value >= 0 && value <= 2) { ctx->up_conversion = value; return MIRA_OK; }
+    if (option == MIRA_OPT_DOWN_SLICES && value >= 0 && value <= 4) { ctx->down_slices_forced = value; return MIRA_OK; }
     if (option == MIRA_OPT_TEST_WAIT_TIMEOUT) { ctx->test_wait_timeout = value != 0; return MIRA_OK; }
     if ((option == MIRA_OPT_HYBRID_MIN_UP || option == MIRA_OPT_HYBRID_MIN_DOWN) && value >= -1) {
         ctx->hybrid_min[option == MIRA_OPT_HYBRID_MIN_UP ? 0 : 1] = value;

@@ -20,6 +20,7 @@
 //
 // Work is derived on the device from the schedule the grouping step wrote; the host never reads
 // routing results.
+#include <algorithm>
 #include "mira_internal.cuh"
 
 namespace mira {
@@ -588,7 +589,8 @@ struct CombineArgs {
     const int32_t* idx; const float* w; const int32_t* perm; const float* ypart;
     const uint32_t* done_mask; uint32_t* miss_mask; int32_t* status;
     void* out; int T, C, k, ns, E, S, out_fp32; long ypart_stride;
-    const int32_t* count; int down_tc_min;      // terms of experts with count >= down_tc_min have one slice (tensor-core down kernel)
+    const int32_t* count; int down_tc_min;      // terms of experts with count >= down_tc_min come from the tensor-core down kernel ...
+    int S_stream, S_tc;                         // ... in this many slices; S = the larger of the two kernels' slice counts in use
 };
 
 constexpr int kCombineThreads = 128;
@@ -610,7 +612,7 @@ __global__ void __launch_bounds__(kCombineThreads) k_combine(CombineArgs A) {
         const bool done = (A.done_mask[e >> 5] >> (e & 31)) & 1u;
         if (!done && blockIdx.x == 0) { atomicOr(A.miss_mask + (e >> 5), 1u << (e & 31)); atomicOr(A.status, 1); }
         s_pos[j] = done ? pos : -1;
-        s_S[j] = (A.count[e] >= A.down_tc_min) ? 1 : A.S;
+        s_S[j] = (A.count[e] >= A.down_tc_min) ? A.S_tc : A.S_stream;
         s_w[j] = wj;
     }
     pdl_wait();            // the routing results above are older than the kernel before this one; the partial sums are not
@@ -712,7 +714,7 @@ mira_status launch_down(mira_ctx* ctx, void* const* slots, const int32_t* slot_m
     return MIRA_OK;
 }
 
-mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, int down_tc_min, void* out, cudaStream_t st) {
+mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, int tc_splits, int down_tc_min, void* out, cudaStream_t st) {
     CombineArgs A;
     A.idx = ws_ptr<int32_t>(ctx, ctx->lay.idx); A.w = ws_ptr<float>(ctx, ctx->lay.w);
     A.perm = ws_ptr<int32_t>(ctx, ctx->lay.perm); A.ypart = ws_ptr<float>(ctx, ctx->lay.ypart);
@@ -720,7 +722,7 @@ mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, int down_tc_
     A.miss_mask = reinterpret_cast<uint32_t*>(A.status) + 16;
     A.done_mask = A.miss_mask + 8;
     A.out = out; A.T = T; A.C = ctx->cfg.hidden; A.k = k; A.ns = ctx->cfg.n_shared; A.E = ctx->cfg.n_experts;
-    A.S = splits; A.out_fp32 = ctx->cfg.out_dtype;
+    A.S_stream = splits; A.S_tc = tc_splits; A.S = std::max(splits, tc_splits); A.out_fp32 = ctx->cfg.out_dtype;
     A.count = ws_ptr<int32_t>(ctx, ctx->lay.count); A.down_tc_min = down_tc_min;
     A.ypart_stride = (long)T * (k + ctx->cfg.n_shared) * ctx->cfg.hidden;
     dim3 grid((ctx->cfg.hidden / 4 + kCombineThreads - 1) / kCombineThreads, T);

@@ -84,6 +84,7 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // that a tile does not start with an empty weight ring: down kernel of the fine-grained layer at 1024 tokens 99 against
 // 102 us, up/gate of the Mixtral shape at 128 tokens 226 against 218 us, nothing elsewhere; the stages already converted
 // cover the restart.)
+constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
 
@@ -102,6 +103,8 @@ struct TcArgs {
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
     int up_conversion;          // up/gate codes: 0, 1 exact conversion; 2 offset subnormals
     uint32_t spin_limit;        // polls after which a barrier wait gives up (kSpinLimit; shortened by MIRA_OPT_TEST_WAIT_TIMEOUT)
+    int down_splits;            // S5, one-CTA layouts: slices of the reduction, each its own tile and its own ypart slice
+    long ypart_stride;          // elements between two slices of ypart
     int drop_first_load;        // test hook: CTA 0 leaves out the activation load of its first K-block, so the waits on that
                                 // stage run out and the kernel leaves through its time-out path
 };
@@ -215,7 +218,7 @@ __device__ __forceinline__ unsigned short f32_to_f16_sat(float v) {
 __device__ __forceinline__ float pow2_f(int e) { return __uint_as_float((unsigned)(max(-126, min(127, e)) + 127) << 23); }
 __device__ __forceinline__ int expo_f(float v) { return (int)((__float_as_uint(v) >> 23) & 0xff) - 127; }
 
-struct Tile { int pos0, ntok, row0, wide; const unsigned char* blob; };
+struct Tile { int pos0, ntok, row0, wide, kb0, nkb, split; const unsigned char* blob; };
 
 // One MMA row's 64 codes of a K-block (shared memory, 64 bytes) -> 32 half2 in k order. SUB: as the fp16
 // subnormals (code + 128) * 2^-24, no subtraction here; else the signed codes, exactly.
@@ -261,6 +264,12 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     const int K = DOWN ? R : C;                       // reduction length
     const int nkb = K / kKB;
     const int n_mb = DOWN ? C / kTileM : R / (kTileM / 2);
+    // S5 may cut the reduction into slices, each a tile of its own whose sums go to its own slice of ypart (the combine
+    // adds the slices in order). The down projection has only C / 128 row tiles, so with few token tiles the CTAs run
+    // a round and a fraction: slices make the rounds shorter. The number of slices depends on the batch size alone,
+    // so every wave of a step uses the same arithmetic.
+    const int S = DOWN ? A.down_splits : 1;
+    const int per_e = n_mb * S;                       // tiles per token tile of an expert (tile counts fit 32 bits: checked by the launcher)
     const size_t per = (size_t)R * C;
 
     const uint32_t b_s = smem_u32(smem);                                          // [stage] B tile
@@ -310,22 +319,30 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const long total = (long)s_ntile[s_nact] * n_mb;
+    const long total = (long)s_ntile[s_nact] * per_e;     // < 2^31
     // Everything above read only what the routing kernels wrote, and those had completed before the kernel in front
     // of this one started (it waited for them before letting this one launch). The activations come from that
     // kernel itself.
     pdl_wait();
     pdl_launch();
 
-    // tile order: (expert, row block, token tile) with the token tile fastest, so CTAs working at the same
+    // tile order: (expert, slice, row block, token tile) with the token tile fastest, so CTAs working at the same
     // time share weight rows through L2
-    auto decode = [&](long tile) {
+    auto decode = [&](long tile_l) {
         Tile t;
+        const int tile = (int)tile_l;
         int lo = 0, hi = s_nact - 1;
-        while (lo < hi) { int mid = (lo + hi + 1) >> 1; if ((long)s_ntile[mid] * n_mb <= tile) lo = mid; else hi = mid - 1; }
+        while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (s_ntile[mid] * per_e <= tile) lo = mid; else hi = mid - 1; }
         const int nt_e = s_ntile[lo + 1] - s_ntile[lo];
-        const long local = tile - (long)s_ntile[lo] * n_mb;
-        const int nb = (int)(local % nt_e), mb = (int)(local / nt_e);
+        const int local = tile - s_ntile[lo] * per_e;
+        const int rest = local / nt_e, nb = local - rest * nt_e;
+        int mb = rest;
+        t.split = 0; t.kb0 = 0; t.nkb = nkb;
+        if (DOWN && S > 1) {
+            t.split = rest / n_mb; mb = rest - t.split * n_mb;
+            t.kb0 = t.split * nkb / S;
+            t.nkb = (t.split + 1) * nkb / S - t.kb0;
+        }
         t.wide = s_wide[lo];
         const int tn = (DOWN && t.wide) ? kTileN / 2 : kTileN;
         t.pos0 = s_off[lo] + nb * tn;
@@ -344,8 +361,9 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
         const uint32_t w_cp = w_g + (lane & 7) * kWRow + (lane >> 3) * 16;   // + stage * kWStage + i * 8 * kWRow
         const uint32_t w_rd = w_g + lane * kWRow;                             // + stage * kWStage + q * 16
         uint32_t gbase = 0;                                                   // K-blocks of this CTA's earlier tiles
-        for (long tile = blockIdx.x; tile < total && !s_abort; tile += gridDim.x, gbase += (uint32_t)nkb) {
+        for (long tile = blockIdx.x; tile < total && !s_abort; tile += gridDim.x) {
             const Tile t = decode(tile);
+            const int nkb = t.nkb;                              // K-blocks of this tile (a slice of the reduction in S5)
             const bool sub = sub_batch && !t.wide;              // offset subnormals or exact codes: per tile, see above
             // source of the row this lane copies in instruction 0 (MMA row 32 gw + (lane & 7)); instruction i is 8 MMA
             // rows further: + 8 rows of W2^ (S5) or + 4 expert-hidden rows of W1^ / W3^ (S4)
@@ -353,7 +371,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
             size_t src_step;
             {
                 const int mrow = gw * 32 + (lane & 7);
-                if (DOWN) { src = t.blob + per + (size_t)(t.row0 + mrow) * R + (lane >> 3) * 16; src_step = (size_t)8 * R; }
+                if (DOWN) { src = t.blob + per + (size_t)(t.row0 + mrow) * R + (lane >> 3) * 16 + (size_t)t.kb0 * kKB; src_step = (size_t)8 * R; }
                 else { src = t.blob + ((mrow & 1) ? 2 * per : 0) + (size_t)(t.row0 + (mrow >> 1)) * C + (lane >> 3) * 16; src_step = (size_t)4 * C; }
             }
             const int kb0 = (int)(((uint32_t)group + kGroups - gbase % kGroups) % kGroups);   // first K-block of this tile that belongs to the group
@@ -394,6 +412,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
             cp_async_wait<0>();
             (void)row;
             if (!ok) break;
+            gbase += (uint32_t)nkb;
         }
     } else if (warp < kTmaWarp) {
         // ------------------------------------------------ epilogue (thread = MMA row = TMEM lane)
@@ -411,6 +430,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 const int c = t.row0 + row;
                 // per-matrix format: the scale of output column c (row c of W2^)
                 const float so = A.per_matrix ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(t.blob + blob_fmt(1, R, C).s_out)[c]) : 1.f;
+                float* yp = A.ypart + (size_t)t.split * A.ypart_stride;
                 auto store = [&](auto wide_c) {       // compiled with and without the second window, chosen per tile
                     constexpr bool kWide = decltype(wide_c)::value;
                     for (int c0 = 0; c0 < ncol; c0 += 32) {
@@ -428,7 +448,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const int n = c0 + j;
-                            if (n < t.ntok) A.ypart[(size_t)(t.pos0 + n) * C + c] = __uint_as_float(v[j]) * (__ldg(A.hscale + t.pos0 + n) * so);
+                            if (n < t.ntok) yp[(size_t)(t.pos0 + n) * C + c] = __uint_as_float(v[j]) * (__ldg(A.hscale + t.pos0 + n) * so);
                         }
                     }
                 };
@@ -453,11 +473,13 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const float a = __uint_as_float(v[2 * jj]), b = __uint_as_float(v[2 * jj + 1]);
-                            const float oa = __shfl_xor_sync(0xffffffffu, a, 1), ob = __shfl_xor_sync(0xffffffffu, b, 1);
+                            // one exchange per pair: the even lane needs its neighbour's G of the even column, the odd lane
+                            // its neighbour's U of the odd column
+                            const float other = __shfl_xor_sync(0xffffffffu, odd ? a : b, 1);
                             const int n = c0 + 2 * jj + odd;
                             const int pc = t.pos0 + min(n, t.ntok - 1);
                             const float xs = __ldg(A.xs_pos + pc);
-                            float ru = odd ? ob : a, rg = odd ? b : oa;
+                            float ru = odd ? other : a, rg = odd ? b : other;
                             if (kSub) {                       // undo the 2^-24 and the +128 offset of the codes
                                 const float off = -128.f * __ldg(A.sum_pos + pc);
                                 ru = fmaf(ru, 16777216.f, off); rg = fmaf(rg, 16777216.f, off);
@@ -500,7 +522,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 const uint32_t box_bytes = (uint32_t)(hi + 1) * kBoxStep * kKB * 2;
                 const bool two = DOWN && t.wide;                                    // second box: the lower window, behind the first
                 bool ok = true;
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int kb = 0; kb < t.nkb; ++kb) {
                     if (!mbar_wait(b_empty(st), ph, &s_abort, A.spin_limit)) { ok = false; break; }
                     if (A.drop_first_load && blockIdx.x == 0 && tile == blockIdx.x && kb == 0) {    // test hook, see TcArgs
                         if (++st == kBStages) { st = 0; ph ^= 1u; }
@@ -509,10 +531,10 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                     const uint32_t dst = b_s + st * kBTileBytes, bar = b_full(st);
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(two ? 2 * box_bytes : box_bytes) : "memory");
                     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-                                 ::"r"(dst), "l"(map), "r"(kb * kKB), "r"(t.pos0), "r"(bar) : "memory");
+                                 ::"r"(dst), "l"(map), "r"((t.kb0 + kb) * kKB), "r"(t.pos0), "r"(bar) : "memory");
                     if (two)
                         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-                                     ::"r"(dst + box_bytes), "l"(map_lo), "r"(kb * kKB), "r"(t.pos0), "r"(bar) : "memory");
+                                     ::"r"(dst + box_bytes), "l"(map_lo), "r"((t.kb0 + kb) * kKB), "r"(t.pos0), "r"(bar) : "memory");
                     if (++st == kBStages) { st = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -537,7 +559,7 @@ __global__ void __launch_bounds__(TC::kThreads, TC::kCtasPerSm) k_ffn_tc(TcArgs 
                 tc_fence_after();
                 const uint32_t d_t = tmem + buf * kTileN;
                 bool ok = true;
-                for (int kb = 0; kb < nkb; ++kb, ++g) {
+                for (int kb = 0; kb < t.nkb; ++kb, ++g) {
                     if (kIssuers == 2 && (int)(g & 1u) != q) continue;
                     const uint32_t sa = g % kAStages, pa = (g / kAStages) & 1u;
                     if (!ready && !mbar_wait(a_full(sa), pa, &s_abort, A.spin_limit)) { ok = false; break; }
@@ -1034,6 +1056,8 @@ TcArgs make_tc_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) 
     A.up_conversion = ctx->up_conversion;
     A.spin_limit = kSpinLimit;
     A.drop_first_load = 0;
+    A.down_splits = 1;
+    A.ypart_stride = (long)ctx->route_T * (ctx->route_k + ctx->cfg.n_shared) * ctx->cfg.hidden;
     return A;
 }
 
@@ -1081,11 +1105,12 @@ static void launch_cfg(mira_ctx* ctx, const TcArgs& A, const unsigned char (*map
 // Estimated cost of a down projection in a 2-CTA layout with tiles of `tn` tokens: the kernel has few row tiles
 // (C / 128), so what counts is how many ROUNDS of tiles its CTAs run, times the cost of a tile relative to a narrow
 // one (a wide tile covers 1.5 times the tokens at 1.3 times the time: 224 K-blocks take 115 us narrow, 150 us wide).
-// Token-tile columns: exact for the shared experts, tokens / tn plus half a ragged tile per expert for the routed ones.
-static double down_cost(const mira_ctx* ctx, int tn, double tile_cost) {
+// Token-tile columns: exact for the shared experts, tokens / tn plus half a ragged tile per expert for the routed ones
+// (at least one per expert that can be routed to).
+static double down_cost(const mira_ctx* ctx, int tn, double tile_cost, int slices = 1) {
     const double T = ctx->route_T, E = ctx->cfg.n_experts, pairs = T * ctx->route_k;
-    const double cols = pairs / tn + 0.5 * std::min(E, pairs) + ctx->cfg.n_shared * std::ceil(T / tn);
-    const double tiles = cols * (ctx->cfg.hidden / kTileM);
+    const double cols = std::max(std::min(E, pairs), pairs / tn + 0.5 * std::min(E, pairs)) + ctx->cfg.n_shared * std::ceil(T / tn);
+    const double tiles = cols * (ctx->cfg.hidden / kTileM) * slices;
     return std::ceil(tiles / (2.0 * ctx->n_sm)) * tile_cost;
 }
 
@@ -1101,8 +1126,46 @@ static void launch_pair(mira_ctx* ctx, const TcArgs& A, cudaStream_t st) {
 }
 static bool pair_shape_ok(const mira_config& c) { return c.ffn % kTileM == 0 && c.hidden % (2 * kTileM) == 0; }
 
+// Layout and number of reduction slices of the down projection of the step last routed. Both follow from the batch
+// size, the top-k and the configuration alone, so every wave of a step gets the same plan (the slices change the
+// order of the additions). Cost model, in K-blocks: rounds of tiles x (K-blocks of a tile x the layout's relative
+// K-block time + 26 for the epilogue and the hand-over of the accumulator, fitted to the times below); a tile of S
+// slices has 1/S of the K-blocks. Measured on the Mixtral shape at 512 tokens (us, down kernel + combine, 1 / 2 / 3 /
+// 4 slices): 240 + 15 / 198 + 18 / 208 + 20 / 233 + 22; Mixtral-8x22B shape at 256 tokens 284 + 14 / 254 + 17; at other
+// sizes (128 to 2048 tokens) slices bring nothing and one is chosen.
+struct DownPlan { int layout, splits; };
+static DownPlan plan_down(const mira_ctx* ctx) {
+    const long avg = (long)ctx->route_T * ctx->route_k / (ctx->cfg.n_experts > 0 ? ctx->cfg.n_experts : 1);
+    DownPlan p;
+    p.layout = ctx->tc_layout;                             // 0 unless a layout is forced (MIRA_OPT_TENSOR_LAYOUT)
+    p.splits = 1;
+    const bool narrow_only = 2 * avg < NarrowTile::kTileN;
+    if (p.layout == 0)
+        // wide only when the estimate is clearly lower: near a tie the narrow layout is the safer one (1536 tokens: 429 / 460)
+        // (with fewer than half a narrow tile of tokens per expert on average no expert fills a wide tile: narrow.
+        // Fine-grained layer, 128 tokens: 39 against 45 us)
+        p.layout = (narrow_only || 0.9 * down_cost(ctx, NarrowTile::kTileN, 1.0) <= down_cost(ctx, WideTile::kTileN, 1.3)) ? 1 : 2;
+    if ((p.layout == 4 || p.layout == 5) && !pair_shape_ok(ctx->cfg)) p.layout = 2;
+    if (p.layout >= 4) return p;                           // the two-SM kernel takes whole reductions
+    const int nkb = ctx->cfg.ffn / kKB;
+    const int max_s = std::min(std::min(ctx->down_splits, kMaxDownSlices), std::max(1, nkb / 16));
+    if (ctx->down_slices_forced > 0) { p.splits = std::min(ctx->down_slices_forced, std::min(ctx->down_splits, nkb)); return p; }
+    if (ctx->tc_layout != 0) return p;                     // a forced layout keeps whole reductions unless slices are forced too
+    auto cost = [&](int tn, double w, int S) { return down_cost(ctx, tn, 1.0, S) * (w * nkb / S + 26.0); };
+    const double w0 = p.layout == 1 ? 1.0 : 1.3;
+    double best = cost(p.layout == 1 ? NarrowTile::kTileN : WideTile::kTileN, w0, 1);
+    for (int S = 2; S <= max_s; ++S)
+        for (int lay = 1; lay <= (narrow_only ? 1 : 2); ++lay) {
+            const double c = cost(lay == 1 ? NarrowTile::kTileN : WideTile::kTileN, lay == 1 ? 1.0 : 1.3, S);
+            if (c < 0.93 * best) { best = c; p.layout = lay; p.splits = S; }     // slices cost partial-sum traffic: only for a clear gain
+        }
+    return p;
+}
+
+int down_tc_slices(const mira_ctx* ctx) { return plan_down(ctx).splits; }
+
 template <bool DOWN>
-static void launch_tc(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps)[128], cudaStream_t st) {
+static void launch_tc(mira_ctx* ctx, TcArgs& A, const unsigned char (*maps)[128], cudaStream_t st) {
     // Up/gate has many row tiles (R / 64), so its time follows the number of tiles: narrow tiles while an expert gets
     // fewer tokens than fill wide ones on average, then wide, and with few experts and many tokens the big layout.
     // The down projection is chosen by the estimated number of rounds (measured on the Mixtral shape, us narrow /
@@ -1110,13 +1173,10 @@ static void launch_tc(mira_ctx* ctx, const TcArgs& A, const unsigned char (*maps
     // picks the faster one in each case).
     const long avg = (long)ctx->route_T * ctx->route_k / (ctx->cfg.n_experts > 0 ? ctx->cfg.n_experts : 1);
     int layout = ctx->tc_layout;                          // 0 unless a layout is forced (MIRA_OPT_TENSOR_LAYOUT)
-    if (layout == 0) {
-        // wide only when the estimate is clearly lower: near a tie the narrow layout is the safer one (1536 tokens: 429 / 460)
-        // (with fewer than half a narrow tile of tokens per expert on average no expert fills a wide tile: narrow.
-        // Fine-grained layer, 128 tokens: 39 against 45 us)
-        if (DOWN) layout = (2 * avg < NarrowTile::kTileN || 0.9 * down_cost(ctx, NarrowTile::kTileN, 1.0) <= down_cost(ctx, WideTile::kTileN, 1.3)) ? 1 : 2;
-        else layout = avg < kWideMinPerExpert ? 1 : (avg >= 256 && ctx->cfg.n_experts <= 16) ? 3 : 2;
+    if (layout == 0 && !DOWN) {
+        layout = avg < kWideMinPerExpert ? 1 : (avg >= 256 && ctx->cfg.n_experts <= 16) ? 3 : 2;
     }
+    if (DOWN) { const DownPlan p = plan_down(ctx); layout = p.layout; A.down_splits = p.splits; }
     if ((layout == 4 || layout == 5) && !pair_shape_ok(ctx->cfg)) layout = DOWN ? 2 : 3;
     if (layout >= 4) launch_pair<DOWN>(ctx, A, st);
     else if (layout == 1) launch_cfg<DOWN, NarrowTile>(ctx, A, maps, st);

@@ -116,6 +116,7 @@ struct mira_ctx {
     bool test_wait_timeout = false;    // the next tcgen05 up/gate launch drops one load and shortens its waits (MIRA_OPT_TEST_WAIT_TIMEOUT)
     int hybrid_min[2] = {-1, -1};      // MIRA_OPT_HYBRID_MIN_UP / _DOWN: -1 = chosen per step, else the pair count from which an
                                        // expert goes to the tcgen05 kernel of that projection (0: all, INT_MAX: none)
+    int down_slices_forced = 0;        // MIRA_OPT_DOWN_SLICES: 0 = chosen per step, else the reduction slices of the tcgen05 down kernel
     int up_conversion = 0;             // tcgen05 up/gate kernel: 0, 1: exact code conversion; 2: offset subnormals (MIRA_OPT_UP_CONVERSION)
     bool prof_on = false;
     size_t prof_used = 0;
@@ -167,7 +168,8 @@ mira_status launch_pool(mira_ctx*, const float* token_scores, int T, int E, floa
 // expert_ffn.cu
 mira_status launch_up_gate(mira_ctx*, void* const* slots, const int32_t* slot_map, cudaStream_t);
 mira_status launch_down(mira_ctx*, void* const* slots, const int32_t* slot_map, cudaStream_t);
-mira_status launch_combine(mira_ctx*, int T, int k, int splits, int down_tc_min, void* out, cudaStream_t);
+mira_status launch_combine(mira_ctx*, int T, int k, int splits, int tc_splits, int down_tc_min, void* out, cudaStream_t);
+int down_tc_slices(const mira_ctx*);     // reduction slices the tensor-core down kernel uses for the step last routed
 // expert_ffn_tc.cu (tcgen05 path for prefill-sized batches)
 bool tc_shape_ok(const mira_config&);
 bool build_tensor_maps(mira_ctx*);

@@ -510,3 +510,54 @@ def test_hybrid_steps_split_the_experts_between_the_kernel_families(shape, mins)
         m.moe_experts(d["x"], slots, slot_map, expert_ids=needed[::2], final_wave=False)
         two = m.moe_experts(d["x"], slots, slot_map, expert_ids=needed[1::2], final_wave=True)
         assert torch.equal(out, two)
+
+
+@pytest.mark.parametrize("layout", [0, 1, 2, 3])
+def test_reduction_slices_of_the_tensor_core_down_kernel(layout):
+    """The tcgen05 down kernel may cut the expert-hidden dimension into slices (tiles of their own, partial sums added
+    by S6 in slice order). Expert width 12352 = 193 K-blocks (uneven thirds and quarters) gives the workspace four
+    partial-sum slices; 1..4 slices are forced in turn on full, ragged and multi-tile experts, one of them a wide-range
+    expert (two fp16 windows). Against the oracle; as waves (bit-identical: the slices are a property of the step);
+    and a hybrid step whose small experts take the streaming down kernel with its own four slices."""
+    def gen(shape, e):
+        w1, w2, w3 = inputs.expert_weights(shape, e)
+        if e == 1:
+            g = np.random.default_rng(100 + e)
+            w1 = w1 * np.exp(2 * g.standard_normal((shape.R, 1))).astype(np.float32)
+        return w1, w2, w3
+    sh = inputs.LayerShape("slices", C=256, R=12352, E=3, k=2, T=330, n_shared=1, zipf_a=1.2, seed=23)
+    b = _binding()
+    for T in (70, 330):
+        wl = Workload(sh, T, gen=gen)
+        d = wl.device_inputs()
+        m = _mira(sh, T, None, out_fp32=True)
+        blobs = m.quantize_experts(d["w1"], d["w2"], d["w3"])
+        slots = b.slot_table(blobs)
+        slot_map = torch.arange(sh.E + sh.n_shared, dtype=torch.int32, device="cuda")
+        res = oracle.moe_layer(wl.x, wl.wr, wl.bias, wl.blobs, sh.R, sh.k, n_shared=sh.n_shared)
+        m.tensor_layout(layout)
+        outs = []
+        for n in (1, 2, 3, 4):
+            m.down_slices(n)
+            out, dbg = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k, debug=True)
+            torch.cuda.synchronize()
+            assert m.poll_status()[0] == 0
+            assert gate_a(out.cpu().numpy(), res["out64"]) <= TOL, f"layout {layout}, T={T}, {n} slices"
+            outs.append(out.clone())
+        assert not torch.equal(outs[0], outs[2])                  # the slices were really taken: another order of additions
+        cnt = dbg["count"].cpu().tolist()
+        needed = [e for e, c in enumerate(cnt) if c > 0]
+        m.down_slices(3)
+        m.route(d["x"], d["wr"], d["bias"], sh.k)
+        m.moe_experts(d["x"], slots, slot_map, expert_ids=needed[::2], final_wave=False)
+        two = m.moe_experts(d["x"], slots, slot_map, expert_ids=needed[1::2], final_wave=True)
+        assert torch.equal(outs[2], two)
+        m.hybrid_min(0, sorted(cnt[:sh.E])[1] + 1)               # the two least-loaded routed experts: streaming down kernel
+        out = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k)
+        torch.cuda.synchronize()
+        assert m.poll_status()[0] == 0
+        assert gate_a(out.cpu().numpy(), res["out64"]) <= TOL
+        m.hybrid_min(-1, -1)
+        m.down_slices(0)                                          # the library's own choice for this batch
+        out = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k)
+        assert gate_a(out.cpu().numpy(), res["out64"]) <= TOL
