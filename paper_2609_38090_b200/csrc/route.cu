@@ -43,49 +43,64 @@ __device__ __forceinline__ void prefetch_rows_l2(const void* W, int row_bytes, i
             asm volatile("prefetch.global.L2 [%0];\n" ::"l"(static_cast<const char*>(W) + (size_t)e * row_bytes + off));
 }
 
-__device__ __forceinline__ void warp_topk(float (&v)[8], int E, int k, int lane, int* out_idx, float* out_val) {
+// The selection runs on 32-bit keys that order like the logits (sign-magnitude floats mapped to unsigned; -0 counts as
+// +0, a NaN ranks below every number), with two hardware warp reductions per selected expert: the largest key, then
+// the lowest index that holds it. Keys: 0 = no candidate (beyond E, or already selected), 1 = NaN, else the logit.
+// SLOTS = values per lane that can be occupied (2 covers 64 experts): this code runs once per token on the critical
+// path of a decode step, where every instruction is fetched cold, so the short form matters.
+__device__ __forceinline__ unsigned topk_key(float v) {
+    if (!(v == v)) return 1u;
+    const unsigned b = __float_as_uint(v + 0.f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float topk_value(unsigned key) {
+    if (key <= 1u) return key ? __uint_as_float(0x7fc00000u) : -INFINITY;
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+// One selection step: returns the winner's index and key to every lane and retires it. With nothing left the result is
+// index 0 with key 0.
+template <int SLOTS>
+__device__ __forceinline__ void topk_step(unsigned (&key)[SLOTS], int lane, int& win_idx, unsigned& win_key) {
+    unsigned bk = 0u;
+#pragma unroll
+    for (int i = 0; i < SLOTS; ++i) bk = max(bk, key[i]);
+    win_key = __reduce_max_sync(0xffffffffu, bk);
+    unsigned cand = 0xffffffffu;
+#pragma unroll
+    for (int i = SLOTS - 1; i >= 0; --i) if (key[i] == win_key) cand = (unsigned)(lane + 32 * i);
+    const unsigned w = __reduce_min_sync(0xffffffffu, win_key ? cand : 0xffffffffu);
+    win_idx = (w == 0xffffffffu) ? 0 : (int)w;
+#pragma unroll
+    for (int i = 0; i < SLOTS; ++i) if (win_key && lane + 32 * i == win_idx) key[i] = 0u;
+}
+
+template <int SLOTS>
+__device__ __forceinline__ void warp_topk_n(const float (&v)[8], int E, int k, int lane, int* out_idx, float* out_val) {
+    unsigned key[SLOTS];
+#pragma unroll
+    for (int i = 0; i < SLOTS; ++i) key[i] = (lane + 32 * i < E) ? topk_key(v[i]) : 0u;
+#pragma unroll 1
     for (int j = 0; j < k; ++j) {
-        float bv = -INFINITY; int bi = 0x7fffffff;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            int e = lane + 32 * i;
-            if (e < E && (v[i] > bv || (v[i] == bv && e < bi))) { bv = v[i]; bi = e; }
-        }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (bi == 0x7fffffff) bi = 0;  // only if every remaining value is NaN / -inf
-#pragma unroll
-        for (int i = 0; i < 8; ++i) if (lane + 32 * i == bi) v[i] = -INFINITY;
-        if (lane == 0) { out_idx[j] = bi; out_val[j] = bv; }
+        int bi; unsigned bk;
+        topk_step<SLOTS>(key, lane, bi, bk);
+        if (lane == 0) { out_idx[j] = bi; out_val[j] = topk_value(bk); }
     }
+}
+__device__ __forceinline__ void warp_topk(float (&v)[8], int E, int k, int lane, int* out_idx, float* out_val) {
+    if (E <= 64) warp_topk_n<2>(v, E, k, lane, out_idx, out_val);
+    else warp_topk_n<8>(v, E, k, lane, out_idx, out_val);
 }
 
 // The same selection with the results spread over the lanes: lane j (< k) returns the j-th selection. Used by the
-// single-CTA routing kernel, where it measures 0.5 us faster than the list (whose arrays live in local memory); in the
-// one-CTA-per-token kernel it measured 2 us slower, so that one keeps the list.
+// single-CTA routing kernel (at most 16 experts: one slot per lane).
 __device__ __forceinline__ void warp_topk_lanes(float (&v)[8], int E, int k, int lane, int& my_idx, float& my_val) {
     my_idx = 0; my_val = -INFINITY;
+    unsigned key[1] = {lane < E ? topk_key(v[0]) : 0u};
+#pragma unroll 1
     for (int j = 0; j < k; ++j) {
-        float bv = -INFINITY; int bi = 0x7fffffff;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            int e = lane + 32 * i;
-            if (e < E && (v[i] > bv || (v[i] == bv && e < bi))) { bv = v[i]; bi = e; }
-        }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (bi == 0x7fffffff) bi = 0;  // only if every remaining value is NaN / -inf
-#pragma unroll
-        for (int i = 0; i < 8; ++i) if (lane + 32 * i == bi) v[i] = -INFINITY;
-        if (lane == j) { my_idx = bi; my_val = bv; }
+        int bi; unsigned bk;
+        topk_step<1>(key, lane, bi, bk);
+        if (lane == j) { my_idx = bi; my_val = topk_value(bk); }
     }
 }
 
@@ -253,6 +268,24 @@ __device__ __forceinline__ void notify_host(const GroupArgs& G, const int* s_cou
     if (threadIdx.x == 0) { __threadfence_system(); *G.host_flag = G.host_seq; }     // the storing thread releases at system scope
 }
 
+// off[e] = sum of count[0..e), off[n] = the total, for n entries in shared memory, by one warp: every lane adds its run
+// of consecutive entries, a shuffle scan over the lanes' sums gives each run its start. Written as short loops: the
+// code runs once per step in one CTA, where instruction fetch costs more than the arithmetic (a thread walking 64
+// entries took 1.3 us, and so did a fully unrolled version of this).
+__device__ __forceinline__ void exclusive_offsets(const int* count, int* off, int n, int lane) {
+    const int per = (n + 31) >> 5, base = lane * per, stop = min(n, base + per);
+    int sum = 0;
+#pragma unroll 1
+    for (int i = base; i < stop; ++i) sum += count[i];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int up = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += up; }
+    int run = incl - sum;
+#pragma unroll 1
+    for (int i = base; i < stop; ++i) { off[i] = run; run += count[i]; }
+    if (lane == 31) off[n] = incl;
+}
+
 // S3 by one CTA in O(pairs): the routed pairs, in (token, choice) order, are cut into one contiguous range per warp.
 // Pass 1 builds each warp's histogram over the experts (32 pairs per step; lanes with the same expert find each
 // other with match.any, the lowest one adds the group's size). An exclusive prefix over the warps turns the
@@ -290,11 +323,7 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
     }
     for (int s = threadIdx.x; s < ns; s += blockDim.x) s_count[E + s] = T;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int a = 0;
-        for (int e = 0; e < E + ns; ++e) { s_off[e] = a; a += s_count[e]; }
-        s_off[E + ns] = a;
-    }
+    if (warp == 0) exclusive_offsets(s_count, s_off, E + ns, lane);
     __syncthreads();
     notify_host(G, s_count, E + ns);
     for (int e = threadIdx.x; e <= E + ns; e += blockDim.x) {
@@ -420,6 +449,72 @@ __device__ __forceinline__ void write_schedule(Sched* sched, const int* tb, cons
     sched->total_tb[0] = au; sched->total_tb[1] = ad;
 }
 
+// The same schedule written by kMaxExperts threads (thread e = expert e; b = its token blocks, 0 if it does not run):
+// five exclusive prefix sums over the experts (rank among the active ones, token blocks and costs of the two streaming
+// kernels), then every active expert writes its own entries. One loop body serves the five sums (the values wait in
+// shared memory), because this code runs once per step and is fetched cold: with 64 experts the serial loop took 3.7
+// us at the very end of the routing kernel, on the critical path of the step.
+// s_tmp: kSchedScratch ints; the calling threads (exactly kMaxExperts) meet at named barrier 1.
+constexpr int kSerialScheduleMax = 16;
+constexpr int kSchedScratch = 5 * kMaxExperts + 5 * (kMaxExperts / 32);
+__device__ __forceinline__ void write_schedule_parallel(Sched* sched, int b, int cnt, int min_up, int min_down, int* s_tmp) {
+    const int e = threadIdx.x, lane = e & 31, warp = e >> 5;
+    constexpr int kW = kMaxExperts / 32;
+    int* s_v = s_tmp;                        // [5][kMaxExperts]: values, then their exclusive prefixes
+    int* s_w = s_tmp + 5 * kMaxExperts;      // [5][kW]: totals of the warps
+    {
+        const int last = b > 0 ? (cnt - (b - 1) * kTokBlock + 7) >> 3 : 1;            // n-tiles of the last block, 1..4
+        const bool up = b > 0 && cnt < min_up, dn = b > 0 && cnt < min_down;          // taken by the streaming kernel of that projection
+        s_v[e] = b > 0 ? 1 : 0;
+        s_v[kMaxExperts + e] = up ? b : 0;
+        s_v[2 * kMaxExperts + e] = dn ? b : 0;
+        s_v[3 * kMaxExperts + e] = up ? (b - 1) * block_cost(0, 4) + block_cost(0, last) : 0;
+        s_v[4 * kMaxExperts + e] = dn ? (b - 1) * block_cost(1, 4) + block_cost(1, last) : 0;
+    }
+#pragma unroll 1
+    for (int q = 0; q < 5; ++q) {
+        const int x = s_v[q * kMaxExperts + e];
+        int incl = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        if (lane == 31) s_w[q * kW + warp] = incl;
+        s_v[q * kMaxExperts + e] = incl - x;          // exclusive within the warp
+    }
+    asm volatile("bar.sync 1, %0;\n" ::"n"(kMaxExperts) : "memory");
+    int before[5];
+#pragma unroll
+    for (int q = 0; q < 5; ++q) before[q] = 0;
+#pragma unroll 1
+    for (int w = 0; w < warp; ++w) {
+#pragma unroll
+        for (int q = 0; q < 5; ++q) before[q] += s_w[q * kW + w];
+    }
+    if (e == 0) { sched->tc_min[0] = min_up; sched->tc_min[1] = min_down; }
+    if (b > 0 || e == kMaxExperts - 1) {
+        // the last thread also writes the closing entry (its own exclusive prefix + its own value = the totals)
+        const int n = s_v[e] + before[0];
+        const int au = s_v[kMaxExperts + e] + before[1], ad = s_v[2 * kMaxExperts + e] + before[2];
+        const int wu = s_v[3 * kMaxExperts + e] + before[3], wd = s_v[4 * kMaxExperts + e] + before[4];
+        if (b > 0) {
+            sched->act_expert[n] = e;
+            sched->tb_prefix[0][n] = au; sched->tb_prefix[1][n] = ad;
+            sched->w_prefix[0][n] = wu; sched->w_prefix[1][n] = wd;
+        }
+        if (e == kMaxExperts - 1) {
+            // totals = this thread's exclusive prefixes plus its own values (recomputed: cheap, and only here)
+            const int last = b > 0 ? (cnt - (b - 1) * kTokBlock + 7) >> 3 : 1;
+            const bool up = b > 0 && cnt < min_up, dn = b > 0 && cnt < min_down;
+            const int nt = n + (b > 0 ? 1 : 0), tu = au + (up ? b : 0), td = ad + (dn ? b : 0);
+            const int cu = wu + (up ? (b - 1) * block_cost(0, 4) + block_cost(0, last) : 0);
+            const int cd = wd + (dn ? (b - 1) * block_cost(1, 4) + block_cost(1, last) : 0);
+            sched->tb_prefix[0][nt] = tu; sched->tb_prefix[1][nt] = td;
+            sched->w_prefix[0][nt] = cu; sched->w_prefix[1][nt] = cd;
+            sched->n_active = nt;
+            sched->total_tb[0] = tu; sched->total_tb[1] = td;
+        }
+    }
+}
+
 // Called by every thread of a CTA of at least kMaxExperts threads. Thread e looks at expert e; a warp covers one word
 // of the masks, so the experts that run and the misses are collected with a ballot and cost one atomic per word
 // (not one per expert on the same word).
@@ -443,7 +538,12 @@ __device__ __forceinline__ void schedule_body(const SchedArgs& S, const int* cou
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, S.tc_min[0], S.tc_min[1]);    // s_tb is 0 for inactive experts
+    if (Etot <= kSerialScheduleMax) {        // few experts: one thread is as fast as the scans (8 experts: 0.5 us)
+        if (threadIdx.x == 0) write_schedule(S.sched, s_tb, count, Etot, S.tc_min[0], S.tc_min[1]);    // s_tb is 0 for inactive experts
+        return;
+    }
+    if (threadIdx.x >= kMaxExperts) return;
+    write_schedule_parallel(S.sched, s_tb[e], e < Etot ? count[e] : 0, S.tc_min[0], S.tc_min[1], s_act);
 }
 
 // S3 for large batches, one CTA; with do_sched also the work schedule of a call that runs every routed expert.
@@ -461,7 +561,7 @@ __global__ void __launch_bounds__(1024) k_group(GroupArgs G, SchedArgs S, int do
 
 __global__ void __launch_bounds__(256) k_schedule(const int32_t* __restrict__ count, int Etot, SchedArgs S) {
     __shared__ int s_tb[kMaxExperts];
-    __shared__ int s_act[kMaxExperts];
+    __shared__ int s_act[kSchedScratch];
     if ((int)blockIdx.x >= S.n_main) { expert_stats(S, blockIdx.x - S.n_main); return; }
     schedule_body(S, count, Etot, s_tb, s_act);
 }
@@ -474,7 +574,8 @@ constexpr int kTokenSmemBytes = 4096;
 inline size_t token_smem(int C, int n_warps, int E) {
     size_t need = (size_t)C * 2;                                                  // the token row
     need = std::max(need, (size_t)n_warps * (size_t)E * 4);                       // the grouping CTA's histograms
-    return std::max(need, (size_t)kTokenSmemBytes);                               // the schedule's scratch
+    need = std::max(need, (size_t)kSchedScratch * 4);                             // the schedule's scratch
+    return std::max(need, (size_t)kTokenSmemBytes);
 }
 
 struct TokenArgs {
@@ -555,7 +656,7 @@ __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, 
         if (lane == 0) s_sc[e] = acc + (A.bias ? A.bias[e] : 0.f);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 32) {                 // warp 1: warp 0 has the top-k to do
         float a = 0.f, b = 0.f;
         for (int i = 0; i < nwarps; ++i) { a += s_red[1][i]; b += s_red[2][i]; }
         A.xscale[t] = sc_dn; A.xnorm[t] = sqrtf(a) * sc_dn; A.xsum[t] = b;
