@@ -94,26 +94,30 @@ __device__ __forceinline__ void load_table(ItemTable& tab, const Sched* __restri
 
 // Units are weighted by the cost of their token block. Returns the first unit at or after cost position x, where
 // x counts cost * units (0 <= x <= total cost * per_tb); monotonic in x, so consecutive CTAs get adjoining ranges.
-__device__ __forceinline__ long unit_at(const ItemTable& tab, unsigned long long x, long per_tb, int w_full) {
+// I: the integer type of unit numbers and cost positions. The launcher takes 32 bits whenever the largest cost
+// position (cost * units * CTAs) fits: 64-bit divisions are long software routines, and this code runs cold at the
+// start of every CTA, where instruction fetch from memory is what it costs.
+template <typename I>
+__device__ __forceinline__ I unit_at(const ItemTable& tab, I x, I per_tb, int w_full) {
     const int n = tab.n_active;
-    if (x >= (unsigned long long)tab.w_prefix[n] * per_tb) return (long)tab.total_tb * per_tb;
+    if (x >= (I)tab.w_prefix[n] * per_tb) return (I)tab.total_tb * per_tb;
     const int xb = (int)(x / per_tb);
     int lo = 0, hi = n - 1;                                // largest a with w_prefix[a] <= xb
     while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tab.w_prefix[mid] <= xb) lo = mid; else hi = mid - 1; }
-    const unsigned long long local = x - (unsigned long long)tab.w_prefix[lo] * per_tb;
+    const I local = x - (I)tab.w_prefix[lo] * per_tb;
     const int ntb = tab.tb_prefix[lo + 1] - tab.tb_prefix[lo];
-    const unsigned long long full_block = (unsigned long long)w_full * per_tb;
-    const unsigned long long full_span = (unsigned long long)(ntb - 1) * full_block;
-    long blk, in_blk;
+    const I full_block = (I)w_full * per_tb;
+    const I full_span = (I)(ntb - 1) * full_block;
+    I blk, in_blk;
     if (local < full_span) {
-        blk = (long)(local / full_block);
-        in_blk = (long)((local - blk * full_block) / w_full);
+        blk = local / full_block;
+        in_blk = (local - blk * full_block) / w_full;
     } else {
         const int w_last = tab.w_prefix[lo + 1] - tab.w_prefix[lo] - (ntb - 1) * w_full;
         blk = ntb - 1;
-        in_blk = (long)((local - full_span) / w_last);
+        in_blk = (local - full_span) / w_last;
     }
-    return ((long)tab.tb_prefix[lo] + blk) * per_tb + in_blk;
+    return ((I)tab.tb_prefix[lo] + blk) * per_tb + in_blk;
 }
 
 struct FfnArgs {
@@ -493,7 +497,7 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
     }
 }
 
-template <bool DOWN>
+template <bool DOWN, typename I>
 __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ ItemTable tab;
@@ -507,20 +511,20 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     load_table(tab, A.sched, DOWN ? 1 : 0);
     const int pair = threadIdx.x >> 6;
     const int S = DOWN ? A.down_splits : 1;
-    const long n_mg = DOWN ? A.C / (16 * kMT) : A.R / (8 * kMT);
-    const long per_tb = n_mg * S;
-    const long total = (long)tab.total_tb * per_tb;
+    const I n_mg = DOWN ? A.C / (16 * kMT) : A.R / (8 * kMT);
+    const I per_tb = n_mg * S;
+    const I total = (I)tab.total_tb * per_tb;
     if (total == 0) { if (DOWN) { pdl_wait(); pdl_launch(); } return; }
-    const unsigned long long cost = (unsigned long long)tab.w_prefix[tab.n_active] * per_tb;
+    const I cost = (I)tab.w_prefix[tab.n_active] * per_tb;
     const int w_full = block_cost(DOWN ? 1 : 0, 4);
-    long u = unit_at(tab, cost * blockIdx.x / gridDim.x, per_tb, w_full);
-    const long u1 = unit_at(tab, cost * (blockIdx.x + 1) / gridDim.x, per_tb, w_full);
+    I u = unit_at<I>(tab, cost * (I)blockIdx.x / (I)gridDim.x, per_tb, w_full);
+    const I u1 = unit_at<I>(tab, cost * (I)(blockIdx.x + 1) / (I)gridDim.x, per_tb, w_full);
     const unsigned sA = (unsigned)__cvta_generic_to_shared(ringA);
 
     // Describes the step that starts at unit v (valid = false past the end of this CTA's range). S5 of a wide-range
     // expert carries two fp16 windows per token, so a block of more than 16 tokens is taken as two steps over the
     // same units: half 0 = its first 16 tokens, half 1 = the rest.
-    auto decode = [&](long v, int half) {
+    auto decode = [&](I v, int half) {
         StepDesc d;
         d.valid = v < u1;
         d.nstep = 0; d.nt = 0; d.active = false; d.blob = nullptr; d.hexp = 0; d.wide = false; d.last_half = true;
@@ -531,11 +535,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
         while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (tab.tb_prefix[mid] <= tbg) lo = mid; else hi = mid - 1; }
         const int e = tab.act_expert[lo];
         const int tb = tbg - tab.tb_prefix[lo];
-        const long rem = v % per_tb;
-        const int mg = (int)(rem % n_mg);
-        d.split = (int)(rem / n_mg);
-        const long left = u1 - v, in_group = n_mg - mg;
-        const long steps = (left + kPairs - 1) / kPairs;
+        const int rem = (int)(v - (I)tbg * per_tb);            // < per_tb = row groups x slices
+        d.split = rem / (int)n_mg;
+        const int mg = rem - d.split * (int)n_mg;
+        const I left = u1 - v, in_group = n_mg - mg;
+        const I steps = (left + kPairs - 1) / kPairs;
         d.nstep = (int)min(in_group, (left + steps - 1) / steps);
         const int cnt = A.count[e];
         d.pos0 = A.offset[e] + tb * kTokBlock;
@@ -694,12 +698,21 @@ FfnArgs make_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) {
     return A;
 }
 
+// Whether every cost position of a step fits 31 bits: cost of all token blocks (at most 32 per block; a step has at
+// most pairs / 32 + experts blocks) x units per block x CTAs.
+bool fits_32(const mira_ctx* ctx, long long per_tb) {
+    const long long pairs = (long long)ctx->route_T * (ctx->route_k + ctx->cfg.n_shared);
+    const long long blocks = pairs / kTokBlock + ctx->cfg.n_experts + ctx->cfg.n_shared;
+    return blocks * 32 * per_tb * (2LL * ctx->n_sm + 1) < (1LL << 31);
+}
+
 }  // namespace
 
 mira_status launch_up_gate(mira_ctx* ctx, void* const* slots, const int32_t* slot_map, cudaStream_t st) {
     FfnArgs A = make_args(ctx, slots, slot_map);
     ProfScope ps(ctx, MIRA_K_UP_GATE, st);
-    MIRA_CUDA_OK(launch_pdl(k_ffn<false>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
+    if (fits_32(ctx, ctx->cfg.ffn / (8 * kMT))) MIRA_CUDA_OK(launch_pdl(k_ffn<false, int>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
+    else MIRA_CUDA_OK(launch_pdl(k_ffn<false, long long>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
     ctx->launches += 1;
     MIRA_CUDA_OK(cudaGetLastError());
     return MIRA_OK;
@@ -708,7 +721,8 @@ mira_status launch_up_gate(mira_ctx* ctx, void* const* slots, const int32_t* slo
 mira_status launch_down(mira_ctx* ctx, void* const* slots, const int32_t* slot_map, cudaStream_t st) {
     FfnArgs A = make_args(ctx, slots, slot_map);
     ProfScope ps(ctx, MIRA_K_DOWN, st);
-    MIRA_CUDA_OK(launch_pdl(k_ffn<true>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
+    if (fits_32(ctx, (long long)(ctx->cfg.hidden / (16 * kMT)) * ctx->down_splits)) MIRA_CUDA_OK(launch_pdl(k_ffn<true, int>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
+    else MIRA_CUDA_OK(launch_pdl(k_ffn<true, long long>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
     ctx->launches += 1;
     MIRA_CUDA_OK(cudaGetLastError());
     return MIRA_OK;
@@ -734,8 +748,10 @@ mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, int tc_split
 }
 
 mira_status set_ffn_attributes() {
-    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
-    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<false, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<true, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<false, long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<true, long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
     return MIRA_OK;
 }
 
