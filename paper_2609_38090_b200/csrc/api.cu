@@ -217,6 +217,7 @@ mira_status mira_create(const mira_config* cfg, void* dev_workspace, size_t work
     if ((s = set_quantize_attributes()) != MIRA_OK) return s;
     MIRA_CUDA_OK(cudaMemset(static_cast<char*>(dev_workspace) + L.status, 0, 32 * sizeof(int32_t)));
     MIRA_CUDA_OK(cudaMemset(static_cast<char*>(dev_workspace) + L.tickets, 0, ((size_t)cfg->max_tokens / 8 + 1) * 4));
+    MIRA_CUDA_OK(cudaMemset(static_cast<char*>(dev_workspace) + L.sched, 0, sizeof(Sched)));   // the up/gate kernel's rehearsal pass reads it before the first schedule is written
     mira_ctx* ctx = new (std::nothrow) mira_ctx();
     if (!ctx) return MIRA_ERR_INVALID_ARG;
     ctx->cfg = *cfg;
