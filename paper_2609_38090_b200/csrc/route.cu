@@ -298,12 +298,27 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
     const int T = G.T, k = G.k, E = G.E, ns = G.ns, kk = k + ns;
     const int P = T * k;
     if (threadIdx.x < 8) G.done_mask[threadIdx.x] = 0u;
-    for (int i = threadIdx.x; i < nwarps * E; i += blockDim.x) s_hist[i] = 0;
-    __syncthreads();
-    const int chunk = ((P + nwarps - 1) / nwarps + 31) & ~31;
-    const int p0 = min(P, warp * chunk), p1 = min(P, p0 + chunk);
-    int* hist = s_hist + warp * E;
     const unsigned lt = (1u << lane) - 1u;
+    // At most 32 pairs (the decode steps of a beam or a small batch): every warp holds all pairs, one per lane, and
+    // counts "its" experts with one ballot each; no histograms, no prefix over the warps, one pass. This is the
+    // step's critical path and is fetched cold, so the short form is worth its own branch (4 tokens x top-4 of 60
+    // experts: 3.8 -> 2 us).
+    const bool few = P <= 32;
+    int e_mine = -1;
+    if (few) {
+        if (lane < P) e_mine = __ldcg(G.idx + lane);
+#pragma unroll 1
+        for (int e = warp; e < E; e += nwarps) {
+            const unsigned m = __ballot_sync(0xffffffffu, e_mine == e);
+            if (lane == 0) s_count[e] = __popc(m);
+        }
+    } else {
+        for (int i = threadIdx.x; i < nwarps * E; i += blockDim.x) s_hist[i] = 0;
+        __syncthreads();
+    }
+    const int chunk = ((P + nwarps - 1) / nwarps + 31) & ~31;
+    const int p0 = few ? 0 : min(P, warp * chunk), p1 = few ? 0 : min(P, p0 + chunk);
+    int* hist = s_hist + warp * E;
     for (int base = p0; base < p1; base += 32) {
         const int p = base + lane;
         const bool valid = p < p1;
@@ -315,11 +330,13 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
         }
         __syncwarp();
     }
-    __syncthreads();
-    for (int e = threadIdx.x; e < E; e += blockDim.x) {
-        int run = 0;
-        for (int w = 0; w < nwarps; ++w) { const int v = s_hist[w * E + e]; s_hist[w * E + e] = run; run += v; }
-        s_count[e] = run;
+    if (!few) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < E; e += blockDim.x) {
+            int run = 0;
+            for (int w = 0; w < nwarps; ++w) { const int v = s_hist[w * E + e]; s_hist[w * E + e] = run; run += v; }
+            s_count[e] = run;
+        }
     }
     for (int s = threadIdx.x; s < ns; s += blockDim.x) s_count[E + s] = T;
     __syncthreads();
@@ -329,6 +346,13 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
     for (int e = threadIdx.x; e <= E + ns; e += blockDim.x) {
         G.offset[e] = s_off[e];
         if (e < E + ns) G.count[e] = s_count[e];
+    }
+    if (few && warp == 0 && lane < P) {      // rank inside the expert = lower lanes with the same expert (token order)
+        const unsigned m = __match_any_sync(P == 32 ? 0xffffffffu : (1u << P) - 1u, e_mine);
+        const int pos = s_off[e_mine] + __popc(m & lt);
+        const int t = lane / k, j = lane - t * k;
+        G.perm[(size_t)t * kk + j] = pos;
+        G.row_token[pos] = t;
     }
     for (int base = p0; base < p1; base += 32) {
         const int p = base + lane;
