@@ -140,7 +140,6 @@ struct FfnArgs {
     int down_splits, down_slice;
     int per_matrix;             // blob format: 0 shared scale, 1 per-matrix scales (see BlobFmt)
     int n_all;                  // routed + shared experts
-    int rehearse;               // up/gate kernel: run the start-up code once before the wait (see k_ffn)
     long ypart_stride;          // elements between two splits = P * C
 };
 
@@ -500,7 +499,7 @@ __device__ __forceinline__ void ffn_step(const FfnArgs& A, const StepDesc& d, Co
     }
 }
 
-template <bool DOWN, typename I>
+template <bool DOWN, typename I, bool REHEARSE = false>
 __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ ItemTable tab;
@@ -569,8 +568,8 @@ __global__ void __launch_bounds__(kThreads, 2) k_ffn(FfnArgs A) {
     StepDesc cur;
     I total = 0;
 #pragma unroll 1
-    for (int pass = (DOWN || !A.rehearse) ? 1 : 0; pass < 2; ++pass) {
-        if (!DOWN && pass == 1) { __syncthreads(); pdl_wait(); pdl_launch(); }
+    for (int pass = REHEARSE ? 0 : 1; pass < 2; ++pass) {
+        if (!DOWN && pass == 1) { if (REHEARSE) __syncthreads(); pdl_wait(); pdl_launch(); }
         load_table(tab, A.sched, DOWN ? 1 : 0);
         total = (I)tab.total_tb * per_tb;
         const I cost = (I)tab.w_prefix[tab.n_active] * per_tb;
@@ -710,7 +709,6 @@ FfnArgs make_args(mira_ctx* ctx, void* const* slots, const int32_t* slot_map) {
     A.down_splits = ctx->down_splits; A.down_slice = ctx->down_slice;
     A.per_matrix = ctx->cfg.format == MIRA_FORMAT_PER_MATRIX;
     A.n_all = ctx->cfg.n_experts + ctx->cfg.n_shared;
-    A.rehearse = ctx->route_T <= 16;
     A.ypart_stride = (long)ctx->route_T * (ctx->route_k + ctx->cfg.n_shared) * ctx->cfg.hidden;
     return A;
 }
@@ -728,7 +726,9 @@ bool fits_32(const mira_ctx* ctx, long long per_tb) {
 mira_status launch_up_gate(mira_ctx* ctx, void* const* slots, const int32_t* slot_map, cudaStream_t st) {
     FfnArgs A = make_args(ctx, slots, slot_map);
     ProfScope ps(ctx, MIRA_K_UP_GATE, st);
-    if (fits_32(ctx, ctx->cfg.ffn / (8 * kMT))) MIRA_CUDA_OK(launch_pdl(k_ffn<false, int>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
+    if (ctx->route_T <= 16 && fits_32(ctx, ctx->cfg.ffn / (8 * kMT)))        // small steps rehearse their start-up code, see k_ffn
+        MIRA_CUDA_OK(launch_pdl(k_ffn<false, int, true>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
+    else if (fits_32(ctx, ctx->cfg.ffn / (8 * kMT))) MIRA_CUDA_OK(launch_pdl(k_ffn<false, int>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
     else MIRA_CUDA_OK(launch_pdl(k_ffn<false, long long>, dim3(ctx->n_sm * 2), dim3(kThreads), kSmemBytes, st, A));
     ctx->launches += 1;
     MIRA_CUDA_OK(cudaGetLastError());
@@ -766,6 +766,7 @@ mira_status launch_combine(mira_ctx* ctx, int T, int k, int splits, int tc_split
 
 mira_status set_ffn_attributes() {
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<false, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<false, int, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<true, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<false, long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_ffn<true, long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemBytes)));

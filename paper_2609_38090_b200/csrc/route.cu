@@ -293,6 +293,7 @@ __device__ __forceinline__ void exclusive_offsets(const int* count, int* off, in
 // same order: rank = the warp's running rank of that expert + the number of lower lanes with the same expert. The
 // order inside an expert is the token order (a stable counting sort), with no atomics.
 // s_hist: nwarps * E ints of scratch.
+template <bool FEW>
 __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int* s_off, int* s_hist) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int T = G.T, k = G.k, E = G.E, ns = G.ns, kk = k + ns;
@@ -303,7 +304,7 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
     // counts "its" experts with one ballot each; no histograms, no prefix over the warps, one pass. This is the
     // step's critical path and is fetched cold, so the short form is worth its own branch (4 tokens x top-4 of 60
     // experts: 3.8 -> 2 us).
-    const bool few = P <= 32;
+    constexpr bool few = FEW;            // chosen at launch: P <= 32
     int e_mine = -1;
     if (few) {
         if (lane < P) e_mine = __ldcg(G.idx + lane);
@@ -576,7 +577,7 @@ __global__ void __launch_bounds__(1024) k_group(GroupArgs G, SchedArgs S, int do
     __shared__ int s_off[kMaxExperts + 1];
     __shared__ int s_hist[kGroupScratch];
     if ((int)blockIdx.x >= S.n_main) { expert_stats(S, blockIdx.x - S.n_main); return; }
-    group_body(G, s_count, s_off, s_hist);
+    group_body<false>(G, s_count, s_off, s_hist);
     if (do_sched) {
         __syncthreads();
         schedule_body(S, s_count, G.E + G.ns, s_off, s_hist);      // s_off and s_hist are free now
@@ -608,6 +609,7 @@ struct TokenArgs {
     unsigned* ticket; int do_sched;
 };
 
+template <bool FEW>
 __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, SchedArgs S) {
     extern __shared__ __align__(16) unsigned char smem[];
     uint4* xs = reinterpret_cast<uint4*>(smem);                        // [C/8]
@@ -709,7 +711,7 @@ __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, 
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    group_body(G, s_count, s_off, reinterpret_cast<int*>(xs));     // the token row is no longer needed
+    group_body<FEW>(G, s_count, s_off, reinterpret_cast<int*>(xs));     // the token row is no longer needed
     if (A.do_sched) {
         __syncthreads();
         schedule_body(S, s_count, E + G.ns, s_off, reinterpret_cast<int*>(xs));   // s_off and xs are free now
@@ -1085,7 +1087,8 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
         SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, k, single ? 1 : T, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_ROUTE, st);
         if (single) MIRA_CUDA_OK(launch_pdl(k_route_small, dim3(1 + n_stat), dim3(kSingleCtaThreads), (size_t)T * C * 2, st, A, G, S));
-        else MIRA_CUDA_OK(launch_pdl(k_route_token, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
+        else if (T * k <= 32) MIRA_CUDA_OK(launch_pdl(k_route_token<true>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
+        else MIRA_CUDA_OK(launch_pdl(k_route_token<false>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));
         ctx->launches += 1;
         if (fused_schedule) *fused_schedule = A.do_sched;
         MIRA_CUDA_OK(cudaGetLastError());
@@ -1137,7 +1140,8 @@ mira_status launch_pool(mira_ctx* ctx, const float* token_scores, int T, int E, 
 mira_status set_route_attributes() {
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_scores, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_scores_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmemMax));
-    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_small, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
     return MIRA_OK;
 }
