@@ -136,6 +136,38 @@ def test_route_ties_and_shared_positions():
     assert np.array_equal(r["perm"].cpu().numpy(), np.concatenate([perm, perm_sh], axis=1))
 
 
+@pytest.mark.parametrize("shape", ["few_experts", "many_experts"])
+@pytest.mark.parametrize("T", [1, 3, 9, 40, 200])
+def test_route_on_signed_zeros_and_masked_experts(shape, T):
+    """The selection works on integer keys derived from the logits: equal logits must tie (lower index wins; biases of
+    -0.0 and +0.0 both give a logit of zero), and experts masked with a bias of -inf must never be chosen while enough
+    finite logits remain. Zero tokens make every logit equal to its bias, so the logits are known exactly; every
+    routing kernel (one CTA, one CTA per token, score + group kernels) is reached by the token counts."""
+    sh = inputs.TINY if shape == "few_experts" else inputs.LayerShape("many", C=128, R=64, E=70, k=6, T=T, n_shared=1, seed=3)
+    wl = Workload(sh, T)
+    x = np.zeros((T, sh.C), dtype=np.float32)
+    bias = np.zeros(sh.E, dtype=np.float32)
+    bias[::2] = -0.0                                   # signed zeros: all tie, ids 0 .. k-1 in order
+    m = _mira(sh, T)
+    xd, wrd = to_bf16_cuda(x), to_bf16_cuda(wl.wr)
+    r = m.route(xd, wrd, torch.from_numpy(bias).cuda(), sh.k)
+    torch.cuda.synchronize()
+    assert np.array_equal(r["idx"].cpu().numpy(), np.tile(np.arange(sh.k), (T, 1)))
+    assert np.allclose(r["w"].cpu().numpy(), 1.0 / sh.k)
+    g = np.random.default_rng(T)
+    bias = g.standard_normal(sh.E).astype(np.float32)
+    masked = g.choice(sh.E, sh.E - sh.k - 1, replace=False)        # k + 1 experts stay selectable
+    bias[masked] = -np.inf
+    r = m.route(xd, wrd, torch.from_numpy(bias).cuda(), sh.k)
+    torch.cuda.synchronize()
+    idx_ref, w_ref, _, _ = oracle.topk_softmax(np.tile(bias.astype(np.float64), (T, 1)), sh.k)
+    assert np.array_equal(r["idx"].cpu().numpy(), idx_ref)
+    assert np.abs(r["w"].cpu().numpy() - w_ref).max() < 1e-6
+    count, offset, perm, perm_sh = oracle.group(idx_ref, sh.E, sh.n_shared)
+    assert np.array_equal(r["count"].cpu().numpy(), count) and np.array_equal(r["offset"].cpu().numpy(), offset)
+    assert np.array_equal(r["perm"].cpu().numpy(), np.concatenate([perm, perm_sh], axis=1))
+
+
 # ---------------------------------------------------------------- S4-S6
 def _check_layer(wl, out_gpu, res, fp32):
     ref = res["out64"]
