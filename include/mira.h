@@ -78,7 +78,8 @@ enum { MIRA_FORMAT_SHARED = 0, MIRA_FORMAT_PER_MATRIX = 1 };
 /* Routing results (Section II-A; grouping is a stable counting sort by expert, tokens ascending).
  * All pointers are device pointers. */
 typedef struct {
-    int32_t* idx;        /* [T][k]   selected experts, best first (ties: lower index)          */
+    int32_t* idx;        /* [T][k]   selected experts, best first (ties: lower index; -0 = +0; a NaN
+                                     logit ranks below every number, -inf included)            */
     float* w;            /* [T][k]   softmax over the k selected logits                        */
     int32_t* count;      /* [E+n_shared]   pairs per expert (shared experts: T)                */
     int32_t* offset;     /* [E+n_shared+1] exclusive prefix sum of count                       */
