@@ -183,7 +183,7 @@ mira_status set_tc_attributes();
 // sizes the streaming kernels win: Mixtral shape 16 tokens 0.231 / 0.240 ms per step, fine-grained 4 tokens 0.055 /
 // 0.057). The down projection switches earlier: its exact conversion costs the streaming kernel more per weight.
 constexpr int kTensorPathMinTokens = 16;    // below, no buffers of the tensor path are laid out
-inline int tc_min_tokens_up(const mira_config& c) { return c.n_experts + c.n_shared > 16 ? 32 : 56; }
+inline int tc_min_tokens_up(const mira_config& c) { return c.n_experts + c.n_shared > 16 ? 20 : 56; }
 inline int tc_min_tokens_down(const mira_config& c) { return c.n_experts + c.n_shared > 16 ? 16 : 40; }
 // Per projection (0 up/gate, 1 down): the pair count from which an expert of a T-token step goes to the tcgen05
 // kernel (0: every expert; INT_MAX: none). The same rule for every wave of a routed batch.
