@@ -186,6 +186,8 @@ k_scores(const __nv_bfloat16* __restrict__ x, int T, int C, const __nv_bfloat16*
     uint4* xs = reinterpret_cast<uint4*>(smem);                       // [kScoreTok][C/8]
     float* sc = reinterpret_cast<float*>(smem + (size_t)kScoreTok * C * 2);  // [kScoreTok][E]
     __shared__ float s_scale[kScoreTok];
+    pdl_wait();            // (a no-op unless launched with programmatic serialization: the routing path of large batches)
+    pdl_launch();
     const int t0 = blockIdx.x * kScoreTok;
     const int nt = min(kScoreTok, T - t0);
     const int c8 = C / 8;
@@ -576,6 +578,8 @@ __global__ void __launch_bounds__(1024) k_group(GroupArgs G, SchedArgs S, int do
     __shared__ int s_count[kMaxExperts];
     __shared__ int s_off[kMaxExperts + 1];
     __shared__ int s_hist[kGroupScratch];
+    pdl_wait();            // the score kernel's selections
+    pdl_launch();
     if ((int)blockIdx.x >= S.n_main) { expert_stats(S, blockIdx.x - S.n_main); return; }
     group_body<false>(G, s_count, s_off, s_hist);
     if (do_sched) {
@@ -954,6 +958,8 @@ k_scores_wide(const __nv_bfloat16* __restrict__ x, int T, int C, const __nv_bflo
     uint4* xs = reinterpret_cast<uint4*>(smem);                       // [kWideTok][C/8]
     __shared__ float s_scale[kWideTok];
     __shared__ int s_last;
+    pdl_wait();            // the previous step's kernels still read the buffers this kernel rewrites
+    pdl_launch();
     const int t0 = blockIdx.x * kWideTok;
     const int nt = min(kWideTok, T - t0);
     const int c8 = C / 8;
@@ -1097,19 +1103,19 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
     {
         ProfScope ps(ctx, MIRA_K_ROUTE, st);
         if (E > kWideExp && wide_scores_smem(C) <= kWideSmemMax)      // several expert groups: the 2-D grid pays (27 against 39 us at 1024 tokens x 60 experts)
-            k_scores_wide<<<dim3((T + kWideTok - 1) / kWideTok, (E + kWideExp - 1) / kWideExp), kWideThreads, wide_scores_smem(C), st>>>(
+            MIRA_CUDA_OK(launch_pdl(k_scores_wide, dim3((T + kWideTok - 1) / kWideTok, (E + kWideExp - 1) / kWideExp), dim3(kWideThreads), wide_scores_smem(C), st,
                 (const __nv_bfloat16*)x, T, C, (const __nv_bfloat16*)w, b, E, rv.logits, x16, xscale, xnorm,
-                ws_ptr<float>(ctx, ctx->lay.xsum), k, rv.idx, rv.w, ws_ptr<unsigned>(ctx, ctx->lay.tickets));
+                ws_ptr<float>(ctx, ctx->lay.xsum), k, rv.idx, rv.w, ws_ptr<unsigned>(ctx, ctx->lay.tickets)));
         else
-            k_scores<<<(T + kScoreTok - 1) / kScoreTok, kScoreThreads, scores_smem(C, E), st>>>(
-                (const __nv_bfloat16*)x, T, C, (const __nv_bfloat16*)w, b, E, rv.logits, x16, xscale, xnorm, ws_ptr<float>(ctx, ctx->lay.xsum), k, rv.idx, rv.w);
+            MIRA_CUDA_OK(launch_pdl(k_scores, dim3((T + kScoreTok - 1) / kScoreTok), dim3(kScoreThreads), scores_smem(C, E), st,
+                (const __nv_bfloat16*)x, T, C, (const __nv_bfloat16*)w, b, E, rv.logits, x16, xscale, xnorm, ws_ptr<float>(ctx, ctx->lay.xsum), k, rv.idx, rv.w));
     }
     {
         // the schedule of a run over all experts comes out of the same launch
         const int do_sched = slot_map != nullptr;
         SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, k, 1, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_GROUP, st);
-        k_group<<<1 + n_stat, 1024, 0, st>>>(G, S, do_sched);
+        MIRA_CUDA_OK(launch_pdl(k_group, dim3(1 + n_stat), dim3(1024), 0, st, G, S, do_sched));
         if (fused_schedule) *fused_schedule = do_sched;
     }
     ctx->launches += 2;
