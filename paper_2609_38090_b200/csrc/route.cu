@@ -591,6 +591,8 @@ __global__ void __launch_bounds__(1024) k_group(GroupArgs G, SchedArgs S, int do
 __global__ void __launch_bounds__(256) k_schedule(const int32_t* __restrict__ count, int Etot, SchedArgs S) {
     __shared__ int s_tb[kMaxExperts];
     __shared__ int s_act[kSchedScratch];
+    pdl_wait();            // the kernels of the wave before still read the schedule this one rewrites
+    pdl_launch();
     if ((int)blockIdx.x >= S.n_main) { expert_stats(S, blockIdx.x - S.n_main); return; }
     schedule_body(S, count, Etot, s_tb, s_act);
 }
@@ -1127,7 +1129,8 @@ mira_status launch_schedule(mira_ctx* ctx, int T, void* const* slots, const int3
                             int all_experts, cudaStream_t st) {
     SchedArgs S = sched_args(ctx, slots, slot_map, all_experts ? nullptr : host_mask, T, ctx->route_k, 1);
     ProfScope ps(ctx, MIRA_K_SCHEDULE, st);
-    k_schedule<<<1 + (slots != nullptr ? Et(ctx->cfg) : 0), 256, 0, st>>>(ws_ptr<int32_t>(ctx, ctx->lay.count), Et(ctx->cfg), S);
+    MIRA_CUDA_OK(launch_pdl(k_schedule, dim3(1 + (slots != nullptr ? Et(ctx->cfg) : 0)), dim3(256), 0, st,
+                            (const int32_t*)ws_ptr<int32_t>(ctx, ctx->lay.count), Et(ctx->cfg), S));
     ctx->launches += 1;
     MIRA_CUDA_OK(cudaGetLastError());
     return MIRA_OK;

@@ -13,6 +13,8 @@ __global__ void __launch_bounds__(kNormThreads) k_residual_rmsnorm(const __nv_bf
                                                                    const __nv_bfloat162* __restrict__ y, int C2, float eps,
                                                                    __nv_bfloat162* __restrict__ out) {
     __shared__ float s_red[kNormThreads / 32];
+    pdl_wait();            // the layer's combine kernel; launched into the same programmatic chain as the layer's kernels,
+    pdl_launch();          // so the next layer's routing kernel is resident when this one ends
     const size_t row = (size_t)blockIdx.x * C2;
     float2 v[kNormMaxPerThread];
     float ss = 0.f;
@@ -49,9 +51,9 @@ extern "C" mira_status mira_residual_rmsnorm(const void* x, const void* moe_out,
     if (!x || !moe_out || !out || T < 0 || hidden < 2 || (hidden & 1) || hidden > 16384) return MIRA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(moe_out) | reinterpret_cast<uintptr_t>(out)) & 3u) return MIRA_ERR_ALIGN;
     if (T == 0) return MIRA_OK;
-    k_residual_rmsnorm<<<T, kNormThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __nv_bfloat162*>(x), static_cast<const __nv_bfloat162*>(moe_out), hidden / 2, eps,
-        static_cast<__nv_bfloat162*>(out));
+    MIRA_CUDA_OK(launch_pdl(k_residual_rmsnorm, dim3(T), dim3(kNormThreads), 0, static_cast<cudaStream_t>(stream),
+                            static_cast<const __nv_bfloat162*>(x), static_cast<const __nv_bfloat162*>(moe_out), hidden / 2, eps,
+                            static_cast<__nv_bfloat162*>(out)));
     MIRA_CUDA_OK(cudaGetLastError());
     return MIRA_OK;
 }
