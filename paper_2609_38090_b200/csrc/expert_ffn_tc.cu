@@ -83,7 +83,10 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // two ring stages, 64 registers per thread -- lost 9 to 20 %. Weight copies running ahead across tile boundaries, so
 // that a tile does not start with an empty weight ring: down kernel of the fine-grained layer at 1024 tokens 99 against
 // 102 us, up/gate of the Mixtral shape at 128 tokens 226 against 218 us, nothing elsewhere; the stages already converted
-// cover the restart.)
+// cover the restart. 64-token tiles with six ring stages instead of four, two CTAs per SM: identical times at 24 to 64
+// tokens (fine-grained 58.2 against 58.3 us), so with one converter group the period is that group's serial chain per
+// K-block, not the depth of the ring; two groups at 64 tokens spill at the 72 registers two CTAs of 14 warps allow
+// (76.8 against 58.4 us).)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
