@@ -86,7 +86,10 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // cover the restart. 64-token tiles with six ring stages instead of four, two CTAs per SM: identical times at 24 to 64
 // tokens (fine-grained 58.2 against 58.3 us), so with one converter group the period is that group's serial chain per
 // K-block, not the depth of the ring; two groups at 64 tokens spill at the 72 registers two CTAs of 14 warps allow
-// (76.8 against 58.4 us).)
+// (76.8 against 58.4 us), and without the spills -- half a row converted and stored at a time, 16-column epilogue chunks --
+// measure 59.7 us: the same. So neither the ring nor the converters set the period of narrow tiles: what fits all of
+// it is a floor of 100 - 110 cycles per tcgen05.mma (M = 128, K = 16) whatever its N up to 192 (per SM and K-block
+// of four MMAs: 440 - 450 cycles at 32 to 128 tokens, 397 at 192 tokens where the arithmetic itself needs 384).)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
