@@ -88,8 +88,13 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // K-block, not the depth of the ring; two groups at 64 tokens spill at the 72 registers two CTAs of 14 warps allow
 // (76.8 against 58.4 us), and without the spills -- half a row converted and stored at a time, 16-column epilogue chunks --
 // measure 59.7 us: the same. So neither the ring nor the converters set the period of narrow tiles: what fits all of
-// it is a floor of 100 - 110 cycles per tcgen05.mma (M = 128, K = 16) whatever its N up to 192 (per SM and K-block
-// of four MMAs: 440 - 450 cycles at 32 to 128 tokens, 397 at 192 tokens where the arithmetic itself needs 384).)
+// it, per SM and K-block of four MMAs, is 440 - 450 cycles at 32 to 128 tokens and 397 at 192 tokens, where the
+// arithmetic itself needs 384. It is not a floor of the tensor pipe: a stand-alone loop of tcgen05.mma (M = 128, K =
+// 16, A from tensor memory) issues one every 51 cycles from one thread at N <= 64 and at the arithmetic rate from
+// N = 128 on (two threads: at the arithmetic rate from N = 64). Clock stamps in the issuing thread: per K-block 260 -
+// 290 cycles for the four MMAs, 75 - 85 for the commit, 80 for the look-ahead test, 60 - 150 in the wait: the thread
+// is busy 560 of the 870 cycles, yet a second issuing thread in the narrow layout made every size 5 - 10 % slower
+// (fine-grained 64 tokens 61.3 against 58.5 us; the turn hand-over costs what the sharing saves).)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
