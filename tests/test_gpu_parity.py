@@ -547,7 +547,7 @@ def test_hybrid_steps_split_the_experts_between_the_kernel_families(shape, mins)
 @pytest.mark.parametrize("layout", [0, 1, 2, 3])
 def test_reduction_slices_of_the_tensor_core_down_kernel(layout):
     """The tcgen05 down kernel may cut the expert-hidden dimension into slices (tiles of their own, partial sums added
-    by S6 in slice order). Expert width 12352 = 193 K-blocks (uneven thirds and quarters) gives the workspace four
+    by S6 in slice order). Expert width 12416 = 194 K-blocks (uneven thirds and quarters) gives the workspace four
     partial-sum slices; 1..4 slices are forced in turn on full, ragged and multi-tile experts, one of them a wide-range
     expert (two fp16 windows). Against the oracle; as waves (bit-identical: the slices are a property of the step);
     and a hybrid step whose small experts take the streaming down kernel with its own four slices."""
@@ -557,7 +557,7 @@ def test_reduction_slices_of_the_tensor_core_down_kernel(layout):
             g = np.random.default_rng(100 + e)
             w1 = w1 * np.exp(2 * g.standard_normal((shape.R, 1))).astype(np.float32)
         return w1, w2, w3
-    sh = inputs.LayerShape("slices", C=256, R=12352, E=3, k=2, T=330, n_shared=1, zipf_a=1.2, seed=23)
+    sh = inputs.LayerShape("slices", C=256, R=12416, E=3, k=2, T=330, n_shared=1, zipf_a=1.2, seed=23)
     b = _binding()
     for T in (70, 330):
         wl = Workload(sh, T, gen=gen)
@@ -593,3 +593,10 @@ def test_reduction_slices_of_the_tensor_core_down_kernel(layout):
         m.down_slices(0)                                          # the library's own choice for this batch
         out = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k)
         assert gate_a(out.cpu().numpy(), res["out64"]) <= TOL
+        if layout == 0:                                           # the two-SM kernel takes whole reductions whatever is forced
+            m.tensor_layout(4)
+            m.down_slices(1)
+            one = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k).clone()
+            m.down_slices(3)
+            three = m.moe_layer(d["x"], d["wr"], d["bias"], slots, slot_map, sh.k)
+            assert torch.equal(one, three) and gate_a(one.cpu().numpy(), res["out64"]) <= TOL
