@@ -302,18 +302,19 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
     const int P = T * k;
     if (threadIdx.x < 8) G.done_mask[threadIdx.x] = 0u;
     const unsigned lt = (1u << lane) - 1u;
-    // At most 32 pairs (the decode steps of a beam or a small batch): every warp holds all pairs, one per lane, and
-    // counts "its" experts with one ballot each; no histograms, no prefix over the warps, one pass. This is the
+    // At most 64 pairs (the decode steps of a beam or a small batch): every warp holds all pairs, up to two per lane,
+    // and counts "its" experts with a ballot per half; no histograms, no prefix over the warps, one pass. This is the
     // step's critical path and is fetched cold, so the short form is worth its own branch (4 tokens x top-4 of 60
     // experts: 3.8 -> 2 us).
-    constexpr bool few = FEW;            // chosen at launch: P <= 32
-    int e_mine = -1;
+    constexpr bool few = FEW;            // chosen at launch: P <= 64
+    int e_mine = -1, e_hi = -1;          // the experts of pairs `lane` and `lane + 32`
     if (few) {
         if (lane < P) e_mine = __ldcg(G.idx + lane);
+        if (lane + 32 < P) e_hi = __ldcg(G.idx + lane + 32);
 #pragma unroll 1
         for (int e = warp; e < E; e += nwarps) {
-            const unsigned m = __ballot_sync(0xffffffffu, e_mine == e);
-            if (lane == 0) s_count[e] = __popc(m);
+            const unsigned m = __ballot_sync(0xffffffffu, e_mine == e), mh = __ballot_sync(0xffffffffu, e_hi == e);
+            if (lane == 0) s_count[e] = __popc(m) + __popc(mh);
         }
     } else {
         for (int i = threadIdx.x; i < nwarps * E; i += blockDim.x) s_hist[i] = 0;
@@ -350,12 +351,31 @@ __device__ __forceinline__ void group_body(const GroupArgs& G, int* s_count, int
         G.offset[e] = s_off[e];
         if (e < E + ns) G.count[e] = s_count[e];
     }
-    if (few && warp == 0 && lane < P) {      // rank inside the expert = lower lanes with the same expert (token order)
-        const unsigned m = __match_any_sync(P == 32 ? 0xffffffffu : (1u << P) - 1u, e_mine);
-        const int pos = s_off[e_mine] + __popc(m & lt);
-        const int t = lane / k, j = lane - t * k;
-        G.perm[(size_t)t * kk + j] = pos;
-        G.row_token[pos] = t;
+    if (few && warp == 0) {                  // rank inside the expert = earlier pairs with the same expert (token order)
+        const int n_lo = min(P, 32), n_hi = P - n_lo;
+        int below = 0;                       // pairs of the first half with the expert of this lane's second-half pair
+        unsigned m = 0;
+        if (lane < n_lo) m = __match_any_sync(n_lo == 32 ? 0xffffffffu : (1u << n_lo) - 1u, e_mine);
+        if (n_hi > 0) {                      // through a few words of shared memory: zero, first half's group sizes, read
+            if (lane < n_hi) s_hist[e_hi] = 0;
+            __syncwarp();
+            if (lane < n_lo && (m & lt) == 0) s_hist[e_mine] = __popc(m);
+            __syncwarp();
+            if (lane < n_hi) below = s_hist[e_hi];
+        }
+        if (lane < n_lo) {
+            const int pos = s_off[e_mine] + __popc(m & lt);
+            const int t = lane / k, j = lane - t * k;
+            G.perm[(size_t)t * kk + j] = pos;
+            G.row_token[pos] = t;
+        }
+        if (lane < n_hi) {
+            const unsigned mh = __match_any_sync(n_hi == 32 ? 0xffffffffu : (1u << n_hi) - 1u, e_hi);
+            const int pos = s_off[e_hi] + below + __popc(mh & lt);
+            const int p = lane + 32, t = p / k, j = p - t * k;
+            G.perm[(size_t)t * kk + j] = pos;
+            G.row_token[pos] = t;
+        }
     }
     for (int base = p0; base < p1; base += 32) {
         const int p = base + lane;
@@ -1095,7 +1115,7 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
         SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, k, single ? 1 : T, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_ROUTE, st);
         if (single) MIRA_CUDA_OK(launch_pdl(k_route_small, dim3(1 + n_stat), dim3(kSingleCtaThreads), (size_t)T * C * 2, st, A, G, S));
-        else if (T * k <= 32) MIRA_CUDA_OK(launch_pdl(k_route_token<true>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
+        else if (T * k <= 64) MIRA_CUDA_OK(launch_pdl(k_route_token<true>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
         else MIRA_CUDA_OK(launch_pdl(k_route_token<false>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));
         ctx->launches += 1;
         if (fused_schedule) *fused_schedule = A.do_sched;
