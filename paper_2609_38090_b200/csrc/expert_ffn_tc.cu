@@ -94,7 +94,11 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // N = 128 on (two threads: at the arithmetic rate from N = 64). Clock stamps in the issuing thread: per K-block 260 -
 // 290 cycles for the four MMAs, 75 - 85 for the commit, 80 for the look-ahead test, 60 - 150 in the wait: the thread
 // is busy 560 of the 870 cycles, yet a second issuing thread in the narrow layout made every size 5 - 10 % slower
-// (fine-grained 64 tokens 61.3 against 58.5 us; the turn hand-over costs what the sharing saves).)
+// (fine-grained 64 tokens 61.3 against 58.5 us; the turn hand-over costs what the sharing saves). Ring stages of two
+// K-blocks for the narrow layout (one wait, one commit and one look-ahead per eight MMAs; built as a template
+// parameter, correct, removed): 58.2 against 58.5 us. Weight requests of 128 contiguous bytes per row (the converters'
+// ring in pairs of K-blocks) instead of 64: Mixtral shape 64 tokens 214.7 against 204.5 us, 2048 tokens up/gate + 1 %,
+// down - 3 %: not the request size either.)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
