@@ -100,6 +100,9 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // ring in pairs of K-blocks) instead of 64: Mixtral shape 64 tokens 214.7 against 204.5 us, 2048 tokens up/gate + 1 %,
 // down - 3 %: not the request size either.)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
+constexpr int kBigMinPerExpert = 640;            // up/gate: ... from which the big layout is used. Re-measured with the exact code conversion (Mixtral
+                                                // shape, us big / wide): 1024 tokens (256 per expert) 695 / 626, 1536 tokens 942 / 873, 2048 tokens 1182 /
+                                                // 1154, 3072 tokens (768 per expert) 1737 / 1785; Mixtral-8x22B shape 1024 tokens 1148 / 991
 constexpr int kWideMinPerExpert = 144;          // up/gate: average routed tokens per expert from which the wide tiles are used (640 tokens
                                                 // over 8 experts: narrow 434, wide 424, big 414 us; 512 tokens: 359 / 380 / 373)
 
@@ -1189,7 +1192,7 @@ static void launch_tc(mira_ctx* ctx, TcArgs& A, const unsigned char (*maps)[128]
     const long avg = (long)ctx->route_T * ctx->route_k / (ctx->cfg.n_experts > 0 ? ctx->cfg.n_experts : 1);
     int layout = ctx->tc_layout;                          // 0 unless a layout is forced (MIRA_OPT_TENSOR_LAYOUT)
     if (layout == 0 && !DOWN) {
-        layout = avg < kWideMinPerExpert ? 1 : (avg >= 256 && ctx->cfg.n_experts <= 16) ? 3 : 2;
+        layout = avg < kWideMinPerExpert ? 1 : (avg >= kBigMinPerExpert && ctx->cfg.n_experts <= 16) ? 3 : 2;
     }
     if (DOWN) { const DownPlan p = plan_down(ctx); layout = p.layout; A.down_splits = p.splits; }
     if ((layout == 4 || layout == 5) && !pair_shape_ok(ctx->cfg)) layout = DOWN ? 2 : 3;
