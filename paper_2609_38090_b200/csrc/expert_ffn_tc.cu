@@ -98,7 +98,10 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // K-blocks for the narrow layout (one wait, one commit and one look-ahead per eight MMAs; built as a template
 // parameter, correct, removed): 58.2 against 58.5 us. Weight requests of 128 contiguous bytes per row (the converters'
 // ring in pairs of K-blocks) instead of 64: Mixtral shape 64 tokens 214.7 against 204.5 us, 2048 tokens up/gate + 1 %,
-// down - 3 %: not the request size either.)
+// down - 3 %: not the request size either. The converter warps taking every other 32-column chunk of the epilogue in
+// the one-accumulator layouts (they wait for the accumulator with the next tile's first weight copies already
+// issued; eight arrivals free it): wide layout, 2048 tokens, up/gate 1137 against 1145 us, narrow layout 4 - 9 %
+// slower at every size: the epilogue's time is not what the other CTA of the SM cannot hide.)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kBigMinPerExpert = 640;            // up/gate: ... from which the big layout is used. Re-measured with the exact code conversion (Mixtral
                                                 // shape, us big / wide): 1024 tokens (256 per expert) 695 / 626, 1536 tokens 942 / 873, 2048 tokens 1182 /
