@@ -635,8 +635,8 @@ struct TokenArgs {
     unsigned* ticket; int do_sched;
 };
 
-template <bool FEW>
-__global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, SchedArgs S) {
+template <bool FEW, int THREADS>
+__global__ void __launch_bounds__(THREADS) k_route_token(TokenArgs A, GroupArgs G, SchedArgs S) {
     extern __shared__ __align__(16) unsigned char smem[];
     uint4* xs = reinterpret_cast<uint4*>(smem);                        // [C/8]
     __shared__ float s_red[3][32];
@@ -701,8 +701,24 @@ __global__ void __launch_bounds__(1024) k_route_token(TokenArgs A, GroupArgs G, 
     const uint4* wg = reinterpret_cast<const uint4*>(A.W);
     for (int e = warp; e < E; e += nwarps) {
         float acc = 0.f;
+        if (THREADS <= 256) {                // few experts, registers to spare: all loads of a 4096-wide row in flight at once
+            for (int i0 = 0; i0 < c8; i0 += 32 * 16) {
+                uint4 wv[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int i = i0 + lane + 32 * j;
+                    wv[j] = i < c8 ? __ldg(wg + (size_t)e * c8 + i) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int i = i0 + lane + 32 * j;
+                    if (i < c8) acc = dot8(wv[j], xs[i], acc);
+                }
+            }
+        } else {
 #pragma unroll 8
-        for (int i = lane; i < c8; i += 32) acc = dot8(__ldg(wg + (size_t)e * c8 + i), xs[i], acc);
+            for (int i = lane; i < c8; i += 32) acc = dot8(__ldg(wg + (size_t)e * c8 + i), xs[i], acc);
+        }
 #pragma unroll
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (lane == 0) s_sc[e] = acc + (A.bias ? A.bias[e] : 0.f);
@@ -1115,8 +1131,13 @@ mira_status launch_route(mira_ctx* ctx, const void* x, int T, const void* w, con
         SchedArgs S = sched_args(ctx, slots, slot_map, nullptr, T, k, single ? 1 : T, quiet_schedule);
         ProfScope ps(ctx, MIRA_K_ROUTE, st);
         if (single) MIRA_CUDA_OK(launch_pdl(k_route_small, dim3(1 + n_stat), dim3(kSingleCtaThreads), (size_t)T * C * 2, st, A, G, S));
-        else if (T * k <= 64) MIRA_CUDA_OK(launch_pdl(k_route_token<true>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));   // a warp per expert and round
-        else MIRA_CUDA_OK(launch_pdl(k_route_token<false>, dim3(T + n_stat), dim3(E > 16 ? 1024 : 256), token_smem(C, E > 16 ? 32 : 8, E), st, A, G, S));
+        else if (E > 16) {                   // a warp per expert and round
+            if (T * k <= 64) MIRA_CUDA_OK(launch_pdl(k_route_token<true, 1024>, dim3(T + n_stat), dim3(1024), token_smem(C, 32, E), st, A, G, S));
+            else MIRA_CUDA_OK(launch_pdl(k_route_token<false, 1024>, dim3(T + n_stat), dim3(1024), token_smem(C, 32, E), st, A, G, S));
+        } else {
+            if (T * k <= 64) MIRA_CUDA_OK(launch_pdl(k_route_token<true, 256>, dim3(T + n_stat), dim3(256), token_smem(C, 8, E), st, A, G, S));
+            else MIRA_CUDA_OK(launch_pdl(k_route_token<false, 256>, dim3(T + n_stat), dim3(256), token_smem(C, 8, E), st, A, G, S));
+        }
         ctx->launches += 1;
         if (fused_schedule) *fused_schedule = A.do_sched;
         MIRA_CUDA_OK(cudaGetLastError());
@@ -1169,8 +1190,10 @@ mira_status launch_pool(mira_ctx* ctx, const float* token_scores, int T, int E, 
 mira_status set_route_attributes() {
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_scores, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_scores_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmemMax));
-    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<true, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<false, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<true, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_token<false, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
     MIRA_CUDA_OK(cudaFuncSetAttribute(k_route_small, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
     return MIRA_OK;
 }
