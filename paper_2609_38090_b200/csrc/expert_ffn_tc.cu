@@ -101,7 +101,10 @@ using NarrowTile = TileCfg<128, 4, 1, 1, 2>;    // two CTAs per SM, deeper ring
 // down - 3 %: not the request size either. The converter warps taking every other 32-column chunk of the epilogue in
 // the one-accumulator layouts (they wait for the accumulator with the next tile's first weight copies already
 // issued; eight arrivals free it): wide layout, 2048 tokens, up/gate 1137 against 1145 us, narrow layout 4 - 9 %
-// slower at every size: the epilogue's time is not what the other CTA of the SM cannot hide.)
+// slower at every size: the epilogue's time is not what the other CTA of the SM cannot hide. 160-token tiles with
+// three ring stages (the most that two CTAs per SM leave room for in tensor memory) against the wide layout's 192 x 2:
+// up/gate 489 against 518 us at 768 tokens, 603 against 630 at 1024, 1129 against 1116 at 2048: the third stage is
+// worth 4 - 5 % where the tile count stays the same and loses where 160-token tiles are more tiles; not kept.)
 constexpr int kMaxDownSlices = 4;               // reduction slices of the tensor-core down projection (see plan_down)
 constexpr int kBigMinPerExpert = 640;            // up/gate: ... from which the big layout is used. Re-measured with the exact code conversion (Mixtral
                                                 // shape, us big / wide): 1024 tokens (256 per expert) 695 / 626, 1536 tokens 942 / 873, 2048 tokens 1182 /
