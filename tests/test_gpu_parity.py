@@ -76,7 +76,7 @@ def test_quantize_and_unpack_bit_exact(src):
 
 
 # ---------------------------------------------------------------- S1-S3
-@pytest.mark.parametrize("T", [1, 5, 16, 33, 100])
+@pytest.mark.parametrize("T", [1, 5, 16, 17, 20, 32, 33, 100])     # 16 / 17 and 32 / 33: the limits of the short grouping paths (32 and 64 pairs)
 def test_route_bit_exact(T):
     sh = inputs.TINY
     wl, d, m, blobs, slots, slot_map = _setup(sh, T)
