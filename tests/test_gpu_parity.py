@@ -413,7 +413,7 @@ def test_host_side_argument_checks():
     assert m.kernel_launches > 0
 
 
-@pytest.mark.parametrize("T", [5, 40, 300])
+@pytest.mark.parametrize("T", [4, 5, 8, 9, 40, 300])
 def test_many_experts_near_the_limits(T):
     """200 routed + 3 shared experts (the library's limit is 256 in total), top-8: routing tables, schedule and
     both expert paths at their widest."""
